@@ -1,0 +1,236 @@
+"""CPU oracle for the Prox decode-time sparse SwiGLU FFN.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+CUDA library is checked against.  It may be imported by the tests, by the
+smoke check and by the benchmark's CPU-baseline leg, and by nothing else; the
+product path never calls it, and it shares no code with the CUDA library.
+
+Everything is written out step by step in the paper's order and notation
+(Sec. 2.1 "SwiGLU Feed-Forward Networks", Sec. 2.2 "Activation Sparsity",
+Sec. 4.1 "Two-Stage Sparse Inference", Sec. 4.2 "Sparsity Allocation between
+Two Stages", Sec. 4.3 "Hardware-Aware Implementation", appendix "Threshold-
+Based Selection and Token-Adaptive Computation").  All sums are accumulated in
+float64; inputs are bf16 values widened exactly.
+
+Storage convention of the arguments (the `nn.Linear` one): W_gate and W_up are
+[d_ff, d_model] arrays whose row j is the weight vector of intermediate
+channel j (column j of the paper's W in R^{d_model x d_ff}); W_down is
+[d_model, d_ff], whose column j is row j of the paper's W_down.
+
+Pins (tests/test_oracle_*.py): dense special case against library matmul and
+library SiLU; Stage 2 against the dense FFN with unselected channels zeroed;
+exact-score mask against a full sort; the allocation tables printed in the
+paper; the paper's closed forms q_Lap, q_G, eta, Corr; the residual bound
+||xW - x_sp W|| <= ||r|| ||W||; the order-preservation condition; quantizer
+invariants; a hand-worked 4x4 example.  The mask and output *values* on random
+inputs have no worked example in the paper: parity unpinned for those beyond
+the properties above.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "bf16_to_f64", "f64_to_bf16_bits", "silu", "dense_ffn", "quantize_proxy",
+    "dequantize", "input_topk", "input_threshold", "input_sparse_projection", "proxy_scores", "channel_topk",
+    "channel_threshold", "stage2", "forward", "forward_batch", "allocate_budget",
+    "sparsity_to_k", "effective_sparsity",
+]
+
+
+# ---------------------------------------------------------------- dtype glue
+def bf16_to_f64(bits) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> float64, exact."""
+    b = np.asarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(v) -> np.ndarray:
+    """float64 -> nearest bf16 (ties to even) bit pattern; via float32 only when
+    that does not introduce a double rounding (checked by construction: the
+    float32 step is exact for values that are already float32)."""
+    v = np.asarray(v, dtype=np.float64)
+    f = v.astype(np.float32)
+    u = f.view(np.uint32)
+    # Repair double rounding: if the f32 rounding moved the value onto a bf16
+    # tie, decide the tie by the sign of the f32 rounding error instead.
+    low = u & np.uint32(0xFFFF)
+    tie = low == np.uint32(0x8000)
+    err = v - f.astype(np.float64)            # >0: true value is above f
+    up = u + np.uint32(0x8000)                # round half up (in magnitude)
+    down = u                                  # truncate (in magnitude)
+    rne = u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))
+    mag_up = (err > 0) == (f >= 0)            # true magnitude is above |f|
+    res = np.where(tie & (err != 0), np.where(mag_up, up, down), rne)
+    return (res >> np.uint32(16)).astype(np.uint16)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    """SiLU(z) = z * sigmoid(z) = z / (1 + exp(-z))  (Sec. 2.1; the paper uses
+    SiLU without restating it, this is its standard definition)."""
+    z = np.asarray(z, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        return z / (1.0 + np.exp(-z))
+
+
+# ------------------------------------------------------------ dense SwiGLU
+def dense_ffn(x, w_gate, w_up, w_down):
+    """FFN(x) = (x W_up  (.)  SiLU(x W_gate)) W_down      (Sec. 2.1, first equation)
+    with u = x W_up, h = SiLU(x W_gate), s = u (.) h.  Returns (y, s)."""
+    x = np.asarray(x, dtype=np.float64)
+    u = np.asarray(w_up, dtype=np.float64) @ x
+    h = silu(np.asarray(w_gate, dtype=np.float64) @ x)
+    s = u * h
+    y = np.asarray(w_down, dtype=np.float64) @ s
+    return y, s
+
+
+# --------------------------------------------------------- proxy quantizer
+def quantize_proxy(w, bits: int, group_size: int):
+    """Symmetric integer proxy of a projection matrix (Sec. 4.3: "symmetric
+    per-row INT4 quantization" of W_up and W_gate).
+
+    One scale per intermediate channel j ("row" of the [d_ff, d_model] storage)
+    and per group of `group_size` consecutive input indices (0 = whole row):
+        a      = max |w|  over the group
+        scale  = fp16( fp32(a) / fp32(qmax) ),     qmax = 2^(bits-1) - 1
+        q      = clamp( rint( fp32(w) / fp32(scale) ), -qmax, +qmax )
+    rint rounds halves to even.  A group whose scale is zero gets q = 0.  These
+    few steps are done in IEEE float32 / float16 (not float64) so that a second
+    implementation can reproduce q and scale bit for bit.
+
+    Returns q int8 [d_ff, d_model] and scale float16 [d_ff, d_model/group]."""
+    if bits not in (4, 8):
+        raise ValueError("bits must be 4 or 8")
+    w = np.asarray(w, dtype=np.float32)
+    d_ff, d_model = w.shape
+    g = d_model if group_size == 0 else group_size
+    if d_model % g:
+        raise ValueError("group_size must divide d_model")
+    qmax = np.float32((1 << (bits - 1)) - 1)
+    wg = w.reshape(d_ff, d_model // g, g)
+    a = np.abs(wg).max(axis=2)
+    scale = (a / qmax).astype(np.float16)
+    s32 = scale.astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        r = wg / s32[:, :, None]
+    q = np.clip(np.rint(r), -qmax, qmax)
+    q = np.where(s32[:, :, None] == 0, np.float32(0), q)
+    return q.reshape(d_ff, d_model).astype(np.int8), scale
+
+
+def dequantize(q, scale, group_size: int) -> np.ndarray:
+    """deq[j, i] = q[j, i] * scale[j, i // group]  in float64."""
+    q = np.asarray(q)
+    d_ff, d_model = q.shape
+    g = d_model if group_size == 0 else group_size
+    s = np.asarray(scale, dtype=np.float64).reshape(d_ff, d_model // g)
+    return (q.astype(np.float64).reshape(d_ff, d_model // g, g) * s[:, :, None]).reshape(d_ff, d_model)
+
+
+# ------------------------------------------------------------ Stage 1 masks
+def input_topk(x, k1: int) -> np.ndarray:
+    """Input mask m_x (Sec. 4.1, first indicator) under the per-token top-k rule
+    of the appendix (m_i = 1[i in TopKIndices(|z|, k)]): the k1 indices of
+    largest |x_i|; equal magnitudes are taken in order of increasing index.
+    Returns the kept indices in increasing order."""
+    mag = np.abs(np.asarray(x, dtype=np.float64))
+    order = np.argsort(-mag, kind="stable")
+    return np.sort(order[:k1]).astype(np.int64)
+
+
+def input_threshold(x, tau_x: float) -> np.ndarray:
+    """Input mask m_x with a fixed layer threshold: [m_x]_i = 1[|x_i| >= tau_x]
+    (Sec. 4.1, first indicator).  Returns kept indices in increasing order."""
+    mag = np.abs(np.asarray(x, dtype=np.float64))
+    return np.nonzero(mag >= tau_x)[0].astype(np.int64)
+
+
+def input_sparse_projection(x, idx, w) -> np.ndarray:
+    """Pi_in(x, W, m) = x_[I(m)] W_[I(m), :]   (Sec. 2.2): only the retained
+    input coordinates contribute.  `w` is stored [d_out, d_in]."""
+    x = np.asarray(x, dtype=np.float64)
+    idx = np.asarray(idx, dtype=np.int64)
+    return np.asarray(w, dtype=np.float64)[:, idx] @ x[idx]
+
+
+def proxy_scores(x, idx_x, deq_gate, deq_up) -> np.ndarray:
+    """u~ = Pi_in(x, W~_up, m_x),  h~ = SiLU(Pi_in(x, W~_gate, m_x)),
+    s~ = u~ (.) h~    (Sec. 4.1, proxy equations).  Returns |s~| per channel."""
+    u_t = input_sparse_projection(x, idx_x, deq_up)
+    h_t = silu(input_sparse_projection(x, idx_x, deq_gate))
+    return np.abs(u_t * h_t)
+
+
+def channel_topk(score, k2: int):
+    """Channel mask m_s (Sec. 4.1, second indicator) under the per-token top-k
+    rule: the k2 channels of largest score, equal scores in order of increasing
+    index.  Returns (selected channels in increasing order, score of the k2-th
+    ranked channel)."""
+    score = np.asarray(score, dtype=np.float64)
+    order = np.argsort(-score, kind="stable")
+    keep = order[:k2]
+    return np.sort(keep).astype(np.int64), float(score[keep[-1]])
+
+
+def channel_threshold(score, tau_s: float) -> np.ndarray:
+    """[m_s]_j = 1[|s~_j| >= tau_s]  (Sec. 4.1, second indicator)."""
+    return np.nonzero(np.asarray(score, dtype=np.float64) >= tau_s)[0].astype(np.int64)
+
+
+# ------------------------------------------------------------------ Stage 2
+def stage2(x, sel, w_gate, w_up, w_down):
+    """u_sp = Pi_out(x, W_up, m_s), h_sp = SiLU(Pi_out(x, W_gate, m_s)),
+    s_sp = u_sp (.) h_sp, y = Pi_in(s_sp, W_down, m_s)   (Sec. 4.1, Stage 2).
+    The dense x and the original weights are used.  Returns (y, s_sp)."""
+    x = np.asarray(x, dtype=np.float64)
+    sel = np.asarray(sel, dtype=np.int64)
+    u_sp = np.asarray(w_up, dtype=np.float64)[sel, :] @ x
+    h_sp = silu(np.asarray(w_gate, dtype=np.float64)[sel, :] @ x)
+    s_sp = u_sp * h_sp
+    y = np.asarray(w_down, dtype=np.float64)[:, sel] @ s_sp
+    return y, s_sp
+
+
+# ------------------------------------------------------------- whole path
+def forward(x, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down):
+    """One token through Stage 1 then Stage 2.  Returns a dict with idx_x,
+    score, sel, threshold (score of the k2-th channel), y."""
+    idx_x = input_topk(x, k1)
+    score = proxy_scores(x, idx_x, deq_gate, deq_up)
+    sel, thr = channel_topk(score, k2)
+    y, s_sp = stage2(x, sel, w_gate, w_up, w_down)
+    return {"idx_x": idx_x, "score": score, "sel": sel, "threshold": thr, "y": y, "s_sp": s_sp}
+
+
+def forward_batch(xs, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down):
+    """Tokens are independent: every token gets its own masks (the paper treats
+    single-batch decoding only)."""
+    return [forward(x, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down) for x in xs]
+
+
+# ---------------------------------------------------------- budget helper
+def effective_sparsity(s1: float, s2: float, alpha: float = 1.0 / 3.0) -> float:
+    """e = 1 - C_Prox / C_Dense = s2 - 2 alpha (1 - s1) / 3   (Sec. 4.2)."""
+    return s2 - 2.0 * alpha * (1.0 - s1) / 3.0
+
+
+def allocate_budget(e: float, alpha: float = 1.0 / 3.0, s_ref: float = 0.7,
+                    s1_min: float = 0.0, s1_max: float = 0.7):
+    """Allocation rule of Sec. 4.2: start from s2 = s_ref and solve the
+    effective-sparsity relation for s1; if s1 leaves [s1_min, s1_max], clamp it
+    to the nearest bound and re-solve the relation for s2."""
+    s2 = s_ref
+    s1 = 1.0 - (s2 - e) * 3.0 / (2.0 * alpha)
+    if s1 < s1_min or s1 > s1_max:
+        s1 = min(max(s1, s1_min), s1_max)
+        s2 = e + 2.0 * alpha * (1.0 - s1) / 3.0
+    return s1, s2
+
+
+def sparsity_to_k(s: float, dim: int) -> int:
+    """Number of kept coordinates for sparsity s: (1 - s) * dim rounded to the
+    nearest integer (halves up), at least 1, at most dim.  The paper says
+    "retains the (1 - rho) d_ff coordinates" without a rounding rule."""
+    k = int(np.floor((1.0 - s) * dim + 0.5))
+    return max(1, min(dim, k))

@@ -1,0 +1,437 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix.
+
+Every test here checks oracle/prox_oracle.py against something that is not the
+oracle itself: library routines (torch float64 matmul / SiLU, numpy sorts),
+values printed in the paper (tests/golden/*.txt), closed forms, invariants, a
+hand-worked example, or brute force on tiny inputs.  CPU only.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import prox_oracle as po
+from paper_2607_27591_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _problem(d_model=256, d_ff=384, n_tok=3, seed=3):
+    wg, wu, wd, x = inputs.make_small(d_model, d_ff, n_tok, seed)
+    return po.bf16_to_f64(wg), po.bf16_to_f64(wu), po.bf16_to_f64(wd), po.bf16_to_f64(x)
+
+
+# ------------------------------------------------------------------ dense pin
+def test_dense_ffn_matches_library_swiglu():
+    """Sec. 2.1 definition, evaluated by torch float64 library ops."""
+    wg, wu, wd, x = _problem()
+    for t in range(x.shape[0]):
+        y, s = po.dense_ffn(x[t], wg, wu, wd)
+        xt = torch.from_numpy(x[t])
+        s_ref = (torch.from_numpy(wu) @ xt) * torch.nn.functional.silu(torch.from_numpy(wg) @ xt)
+        y_ref = torch.from_numpy(wd) @ s_ref
+        np.testing.assert_allclose(s, s_ref.numpy(), rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(y, y_ref.numpy(), rtol=1e-11, atol=1e-14)
+
+
+def test_k2_equal_dff_is_dense():
+    """At 0% channel sparsity the whole path equals the dense FFN, whatever the
+    proxy says (proxy values never propagate, Sec. 3.2 / 4.1)."""
+    wg, wu, wd, x = _problem()
+    qg, sg = po.quantize_proxy(wg, 4, 0)
+    qu, su = po.quantize_proxy(wu, 4, 0)
+    dg, du = po.dequantize(qg, sg, 0), po.dequantize(qu, su, 0)
+    d_ff = wg.shape[0]
+    for t in range(x.shape[0]):
+        out = po.forward(x[t], 40, d_ff, dg, du, wg, wu, wd)
+        xt = torch.from_numpy(x[t])
+        y_ref = torch.from_numpy(wd) @ ((torch.from_numpy(wu) @ xt) *
+                                        torch.nn.functional.silu(torch.from_numpy(wg) @ xt))
+        assert np.array_equal(out["sel"], np.arange(d_ff))
+        np.testing.assert_allclose(out["y"], y_ref.numpy(), rtol=1e-11, atol=1e-14)
+
+
+def test_stage2_is_dense_with_unselected_channels_zeroed():
+    """y = Pi_in(s_sp, W_down, m_s) = sum_{j in mask} s_j W_down[j,:]  (Sec. 3.1
+    weighted-sum view, Sec. 4.1 Stage 2)."""
+    wg, wu, wd, x = _problem(seed=5)
+    rng = np.random.default_rng(0)
+    d_ff = wg.shape[0]
+    for t in range(x.shape[0]):
+        sel = np.sort(rng.choice(d_ff, size=97, replace=False))
+        y, s_sp = po.stage2(x[t], sel, wg, wu, wd)
+        xt = torch.from_numpy(x[t])
+        s_full = (torch.from_numpy(wu) @ xt) * torch.nn.functional.silu(torch.from_numpy(wg) @ xt)
+        m = torch.zeros(d_ff, dtype=torch.float64)
+        m[torch.from_numpy(sel)] = 1.0
+        y_ref = torch.from_numpy(wd) @ (s_full * m)
+        np.testing.assert_allclose(y, y_ref.numpy(), rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(s_sp, s_full.numpy()[sel], rtol=1e-12, atol=1e-15)
+        # weighted-sum form, one row of W_down per channel, summed one by one
+        y_rows = np.zeros_like(y)
+        for c, j in enumerate(sel):
+            y_rows += s_sp[c] * wd[:, j]
+        np.testing.assert_allclose(y, y_rows, rtol=1e-10, atol=1e-13)
+
+
+def test_output_depends_on_proxy_only_through_mask():
+    """Two different proxies that give the same mask give bit-identical y."""
+    wg, wu, wd, x = _problem(seed=7)
+    dg4 = po.dequantize(*po.quantize_proxy(wg, 4, 0), 0)
+    du4 = po.dequantize(*po.quantize_proxy(wu, 4, 0), 0)
+    out = po.forward(x[0], 77, 120, dg4, du4, wg, wu, wd)
+    y_again, _ = po.stage2(x[0], out["sel"], wg, wu, wd)
+    assert np.array_equal(out["y"], y_again)
+
+
+# ------------------------------------------------------------ selection pins
+def test_exact_scores_mask_is_full_sort_topk():
+    """oracle-s selection (Sec. 3.1): with exact scores (unquantized weights,
+    all inputs kept) the mask is the (1-rho) d_ff largest |s|."""
+    wg, wu, wd, x = _problem(seed=11)
+    d_model, d_ff = wg.shape[1], wg.shape[0]
+    for t in range(x.shape[0]):
+        for k2 in (1, 13, 128, d_ff - 1, d_ff):
+            out = po.forward(x[t], d_model, k2, wg, wu, wg, wu, wd)
+            _, s = po.dense_ffn(x[t], wg, wu, wd)
+            # brute force: python sort of (magnitude desc, index asc) pairs
+            ranked = sorted(range(d_ff), key=lambda j: (-abs(s[j]), j))[:k2]
+            assert sorted(ranked) == out["sel"].tolist()
+            assert len(out["sel"]) == k2 == len(set(out["sel"].tolist()))
+            assert out["threshold"] == abs(s[ranked[-1]])
+
+
+def test_topk_tie_rule_on_handmade_ties():
+    """Equal magnitudes: lower index wins; exactly k are kept."""
+    z = np.array([1.0, -2.0, 2.0, 0.5, -2.0, 1.0, 0.0, -0.0, 2.0, 1.0])
+    assert po.input_topk(z, 1).tolist() == [1]
+    assert po.input_topk(z, 2).tolist() == [1, 2]
+    assert po.input_topk(z, 3).tolist() == [1, 2, 4]
+    assert po.input_topk(z, 5).tolist() == [0, 1, 2, 4, 8]
+    assert po.input_topk(z, 6).tolist() == [0, 1, 2, 4, 5, 8]
+    assert po.input_topk(z, 9).tolist() == [0, 1, 2, 3, 4, 5, 6, 8, 9]
+    sel, thr = po.channel_topk(np.abs(z), 5)
+    assert sel.tolist() == [0, 1, 2, 4, 8] and thr == 1.0
+    # brute force over every k on random tied data
+    rng = np.random.default_rng(1)
+    v = rng.integers(0, 4, size=16).astype(np.float64)
+    for k in range(1, 17):
+        want = sorted(sorted(range(16), key=lambda i: (-v[i], i))[:k])
+        assert po.channel_topk(v, k)[0].tolist() == want
+        assert po.input_topk(-v, k).tolist() == want
+
+
+def test_threshold_rule_keeps_all_at_or_above_tau():
+    z = np.array([0.5, -1.0, 1.0, 0.99, -3.0])
+    assert po.input_threshold(z, 1.0).tolist() == [1, 2, 4]
+    assert po.channel_threshold(np.abs(z), 0.99).tolist() == [1, 2, 3, 4]
+
+
+def test_topk_minimises_residual_energy_bruteforce():
+    """Sec. 3.2: keeping the largest magnitudes minimises ||r||_2 over all
+    coordinate-sparse approximations of the same density (all subsets, tiny d)."""
+    import itertools
+    rng = np.random.default_rng(2)
+    x = rng.laplace(size=9)
+    for k in (1, 3, 5, 8):
+        kept = po.input_topk(x, k)
+        best = min(itertools.combinations(range(9), k),
+                   key=lambda c: np.sum(np.delete(x, list(c)) ** 2))
+        assert sorted(best) == kept.tolist()
+
+
+# ----------------------------------------------------------- hand-worked pin
+def _read_hand():
+    rows = {}
+    for line in open(os.path.join(GOLDEN, "hand_worked_4x4.txt")):
+        line = line.split("#")[0].strip()
+        if line:
+            k, *v = line.split()
+            rows[k] = [float(t) for t in v]
+    return rows
+
+
+def test_hand_worked_example():
+    g = _read_hand()
+    x = np.array(g["x"])
+    wg = np.array([g[f"w_gate{j}"] for j in range(4)])
+    wu = np.array([g[f"w_up{j}"] for j in range(4)])
+    wd = np.array([g[f"w_down{d}"] for d in range(4)])
+    qg, sg = po.quantize_proxy(wg, 4, 0)
+    qu, su = po.quantize_proxy(wu, 4, 0)
+    assert np.array_equal(qg, np.array([g[f"q_gate{j}"] for j in range(4)], dtype=np.int8))
+    assert np.all(sg.astype(np.float64) == 0.125) and np.all(su.astype(np.float64) == 0.125)
+    dg, du = po.dequantize(qg, sg, 0), po.dequantize(qu, su, 0)
+    assert np.array_equal(dg, wg) and np.array_equal(du, wu)
+    idx = po.input_topk(x, 2)
+    assert idx.tolist() == [int(v) for v in g["idx_x"]]
+    gp = po.input_sparse_projection(x, idx, dg)
+    up = po.input_sparse_projection(x, idx, du)
+    assert gp.tolist() == g["g_proxy"] and up.tolist() == g["u_proxy"]
+    score = po.proxy_scores(x, idx, dg, du)
+    want = [abs(u * z / (1.0 + math.exp(-z))) for u, z in zip(g["u_proxy"], g["g_proxy"])]
+    np.testing.assert_allclose(score, want, rtol=1e-15)
+    np.testing.assert_allclose(score, [4.4506, 0.3557, 0.4216, 1.1182], atol=5e-5)
+    sel, thr = po.channel_topk(score, 2)
+    assert sel.tolist() == [int(v) for v in g["sel"]]
+    y, s_sp = po.stage2(x, sel, wg, wu, wd)
+    s_want = [u * z / (1.0 + math.exp(-z)) for u, z in zip(g["u_exact"], g["g_exact"])]
+    np.testing.assert_allclose(s_sp, s_want, rtol=1e-15)
+    y_want = [sum(s_want[c] * g[f"w_down{d}"][j] for c, j in enumerate(sel)) for d in range(4)]
+    np.testing.assert_allclose(y, y_want, rtol=1e-14)
+    np.testing.assert_allclose(y, [-1.227494, -3.502545, -0.523779, 3.764435], atol=2e-6)
+    full = po.forward(x, 2, 2, dg, du, wg, wu, wd)
+    assert np.array_equal(full["y"], y) and full["sel"].tolist() == sel.tolist()
+
+
+# ------------------------------------------------------------ quantizer pins
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0), (8, 128)])
+def test_quantizer_invariants(bits, group):
+    wg, _, _, _ = _problem(d_model=256, d_ff=96, seed=13)
+    wg[5, :] = 0.0                       # an all-zero row
+    wg[6, 128:] = 0.0                    # an all-zero group
+    q, scale = po.quantize_proxy(wg, bits, group)
+    qmax = 2 ** (bits - 1) - 1
+    g = wg.shape[1] if group == 0 else group
+    assert q.dtype == np.int8 and scale.dtype == np.float16
+    assert scale.shape == (wg.shape[0], wg.shape[1] // g)
+    assert np.abs(q).max() <= qmax
+    deq = po.dequantize(q, scale, group)
+    s_full = np.repeat(scale.astype(np.float64), g, axis=1)
+    assert np.all(np.abs(wg - deq) <= 0.5 * s_full * (1 + 1e-6) + 1e-30)
+    qg = np.abs(q).reshape(wg.shape[0], -1, g).max(axis=2)
+    nz = scale.astype(np.float64) > 0
+    assert np.all(qg[nz] == qmax) and np.all(qg[~nz] == 0)
+    assert np.all(q[5] == 0) and np.all(scale[5] == 0)
+    if group:
+        assert np.all(q[6, 128:] == 0) and scale[6, 1] == 0
+    # re-quantizing the dequantized matrix is the identity on q
+    q2, scale2 = po.quantize_proxy(deq, bits, group)
+    assert np.array_equal(q2, q) and np.array_equal(scale2, scale)
+    # sign symmetry
+    qn, sn = po.quantize_proxy(-wg, bits, group)
+    assert np.array_equal(qn, -q) and np.array_equal(sn, scale)
+
+
+def test_quantizer_exact_rational_check():
+    """Brute-force check of rint(w / scale) with exact rationals on a small
+    matrix: the float32 division must round to the integer nearest to the exact
+    quotient (ties to even), which a float32 quotient guarantees for |q| <= 127."""
+    rng = np.random.default_rng(17)
+    w = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(
+        (rng.standard_normal((8, 64)) * 0.02).astype(np.float32))).astype(np.float64)
+    for bits in (4, 8):
+        q, scale = po.quantize_proxy(w, bits, 0)
+        qmax = 2 ** (bits - 1) - 1
+        for j in range(8):
+            sc = Fraction(float(scale[j, 0]))
+            # scale itself: fp16 nearest to fp32(a)/fp32(qmax)
+            a32 = np.float32(np.abs(w[j]).max())
+            assert scale[j, 0] == np.float16(np.float32(a32 / np.float32(qmax)))
+            for i in range(64):
+                exact = Fraction(float(w[j, i])) / sc
+                near = round(exact)          # python rounds halves to even
+                # float32 quotient can only differ from `exact` by < 2^-24 rel;
+                # exclude the measure-zero case of straddling a half
+                if abs(exact - near) < Fraction(1, 2) - Fraction(1, 10 ** 5):
+                    assert q[j, i] == max(-qmax, min(qmax, near))
+
+
+def test_int8_proxy_ranks_closer_to_exact_than_int4():
+    wg, wu, wd, x = _problem(d_model=512, d_ff=1024, n_tok=4, seed=19)
+    d_model, d_ff = 512, 1024
+    ov = {}
+    for bits in (4, 8):
+        dg = po.dequantize(*po.quantize_proxy(wg, bits, 0), 0)
+        du = po.dequantize(*po.quantize_proxy(wu, bits, 0), 0)
+        tot = 0
+        for t in range(x.shape[0]):
+            a = po.forward(x[t], d_model, 256, dg, du, wg, wu, wd)["sel"]
+            b = po.forward(x[t], d_model, 256, wg, wu, wg, wu, wd)["sel"]
+            tot += len(set(a.tolist()) & set(b.tolist()))
+        ov[bits] = tot
+    assert ov[8] > ov[4] > 0.8 * 4 * 256
+
+
+def test_proxy_storage_is_one_sixth_of_ffn_bytes():
+    """Sec. 6 (limitations): INT4 proxies add about 12% weight storage.  Two
+    INT4 matrices against three bf16 ones: 2*(1/2) / (3*2) = 1/6 of the FFN;
+    with FFNs at roughly 70-75% of model parameters that is 12%."""
+    d_model, d_ff = 4096, 12288
+    proxy = 2 * d_model * d_ff * 4 // 8
+    ffn = 3 * d_model * d_ff * 2
+    assert Fraction(proxy, ffn) == Fraction(1, 6)
+    assert 0.11 < (1 / 6) * 0.72 < 0.13
+
+
+# ------------------------------------------------------------- budget pins
+def _alloc_rows():
+    for line in open(os.path.join(GOLDEN, "stagewise_allocation.txt")):
+        line = line.split("#")[0].strip()
+        if line:
+            src, e, cap, s1, s2 = line.split()
+            yield src, float(e) / 100, float(cap) / 100, (None if s1 == "-" else float(s1) / 100), float(s2)
+
+
+def test_allocation_tables_printed_in_paper():
+    n = 0
+    for src, e, cap, s1_want, s2_want in _alloc_rows():
+        s1, s2 = po.allocate_budget(e, alpha=1 / 3, s_ref=0.7, s1_min=0.0, s1_max=cap)
+        assert f"{100 * s2:.1f}" == f"{s2_want:.1f}", (src, e, cap)
+        if s1_want is not None:
+            assert abs(s1 - s1_want) < 1e-9
+        assert abs(po.effective_sparsity(s1, s2) - e) < 1e-12      # Sec. 4.2 relation
+        n += 1
+    assert n == 10
+
+
+def test_cost_model_relation():
+    """e = 1 - C_Prox / C_Dense with C_Prox = 2 alpha (1 - s1) + 3 (1 - s2), C_Dense = 3."""
+    for s1, s2, a in ((0.7, 0.7667, 1 / 3), (0.0, 0.622, 1 / 3), (0.3, 0.8, 0.285)):
+        c = 2 * a * (1 - s1) + 3 * (1 - s2)
+        assert abs(po.effective_sparsity(s1, s2, a) - (1 - c / 3)) < 1e-15
+
+
+def test_workload_budgets_follow_allocation_rule():
+    for wl in inputs.WORKLOADS.values():
+        for e, (k1, k2) in wl.points.items():
+            s1, s2 = po.allocate_budget(e / 100)
+            assert po.sparsity_to_k(s1, wl.d_model) == k1, (wl.name, e)
+            assert po.sparsity_to_k(s2, wl.d_ff) == k2, (wl.name, e)
+            # realised sparsity equals the target up to rounding of k
+            e_hat = po.effective_sparsity(1 - k1 / wl.d_model, 1 - k2 / wl.d_ff)
+            assert abs(e_hat - e / 100) < 1.0 / wl.d_model + 1.0 / wl.d_ff
+    sweep = inputs.WORKLOADS["llama3_70b"].extra["s1_sweep"]
+    for n, (k1, k2) in enumerate(sweep):
+        s1 = n / 10
+        s2 = 0.7 + 2 * (1 / 3) * (1 - s1) / 3
+        assert (po.sparsity_to_k(s1, 8192), po.sparsity_to_k(s2, 28672)) == (k1, k2)
+
+
+def test_sparsity_to_k_edges():
+    assert po.sparsity_to_k(0.0, 100) == 100
+    assert po.sparsity_to_k(1.0, 100) == 1
+    assert po.sparsity_to_k(0.995, 100) == 1       # 0.5 rounds up
+    assert po.sparsity_to_k(0.985, 100) == 2
+    assert po.sparsity_to_k(-0.5, 100) == 100
+
+
+# -------------------------------------------------------- closed-form pins
+def _closed():
+    out = {}
+    for line in open(os.path.join(GOLDEN, "closed_forms.txt")):
+        line = line.split("#")[0].strip()
+        if line:
+            name, p, v, _ = line.split()
+            out[name] = (float(p), float(v))
+    return out
+
+
+def test_laplace_energy_kept_by_magnitude_topk():
+    """q_Lap(0.7) ~ 0.879: top-30% magnitudes of Laplace samples keep ~87.9% of
+    the energy.  Pins the magnitude top-k rule statistically."""
+    p, want = _closed()["q_lap"]
+    a = -math.log(1 - p)
+    assert abs((1 - p) / 2 * (a * a + 2 * a + 2) - want) < 5e-4
+    rng = np.random.default_rng(23)
+    z = rng.laplace(0, 1.7, size=200_000)
+    kept = po.input_topk(z, po.sparsity_to_k(p, z.size))
+    frac = np.sum(z[kept] ** 2) / np.sum(z ** 2)
+    assert abs(frac - want) < 6e-3
+    # the complement rule (keep the smallest) would keep ~12% - far outside
+    assert frac > 0.85
+
+
+def test_gaussian_input_sparse_projection_error_and_correlation():
+    """q_G(0.7) ~ 0.783, eta ~ 0.465, Corr ~ 0.885 for Gaussian x and iid
+    Gaussian weights.  Pins Pi_in together with the kept-largest rule."""
+    c = _closed()
+    p = c["q_g"][0]
+    rng = np.random.default_rng(29)
+    d_in, d_out = 4096, 1536
+    w = rng.standard_normal((d_out, d_in))
+    q_acc, eta_acc, corr_acc, n = 0.0, 0.0, 0.0, 6
+    for _ in range(n):
+        x = rng.standard_normal(d_in) * 0.8
+        idx = po.input_topk(x, po.sparsity_to_k(p, d_in))
+        dense = w @ x
+        sp = po.input_sparse_projection(x, idx, w)
+        q_acc += np.sum(x[idx] ** 2) / np.sum(x ** 2)
+        eta_acc += np.linalg.norm(dense - sp) / np.linalg.norm(dense)
+        corr_acc += np.corrcoef(dense, sp)[0, 1]
+    assert abs(q_acc / n - c["q_g"][1]) < 0.01
+    assert abs(eta_acc / n - c["eta"][1]) < 0.015
+    assert abs(corr_acc / n - c["corr"][1]) < 0.012
+
+
+def test_residual_bound():
+    """||x W - x_sp W||_2 <= ||r||_2 ||W||_2   (Sec. 3.2)."""
+    wg, wu, wd, x = _problem(d_model=256, d_ff=384, seed=31)
+    spec = np.linalg.norm(wg, 2)
+    for t in range(x.shape[0]):
+        for k in (1, 26, 77, 255):
+            idx = po.input_topk(x[t], k)
+            r = x[t].copy()
+            r[idx] = 0.0
+            lhs = np.linalg.norm(wg @ x[t] - po.input_sparse_projection(x[t], idx, wg))
+            assert lhs <= np.linalg.norm(r) * spec * (1 + 1e-12)
+            np.testing.assert_allclose(lhs, np.linalg.norm(wg @ r), rtol=1e-9)
+
+
+def test_order_preserved_when_gap_exceeds_perturbation():
+    """If s~_i = s_i + delta_i, the order of |s_i|, |s_j| is kept whenever
+    ||s_i| - |s_j|| > |delta_i| + |delta_j|  (appendix, ranking preservation)."""
+    wg, wu, wd, x = _problem(d_model=256, d_ff=384, seed=37)
+    dg = po.dequantize(*po.quantize_proxy(wg, 4, 0), 0)
+    du = po.dequantize(*po.quantize_proxy(wu, 4, 0), 0)
+    for t in range(x.shape[0]):
+        idx = po.input_topk(x[t], 77)
+        s_t = po.input_sparse_projection(x[t], idx, du) * po.silu(po.input_sparse_projection(x[t], idx, dg))
+        _, s = po.dense_ffn(x[t], wg, wu, wd)
+        delta = np.abs(s_t - s)
+        gap = np.abs(np.abs(s)[:, None] - np.abs(s)[None, :])
+        safe = gap > delta[:, None] + delta[None, :]
+        same = (np.abs(s)[:, None] > np.abs(s)[None, :]) == (np.abs(s_t)[:, None] > np.abs(s_t)[None, :])
+        assert safe.sum() > 0 and np.all(same[safe])
+        np.testing.assert_array_equal(np.abs(s_t), po.proxy_scores(x[t], idx, dg, du))
+
+
+# ---------------------------------------------------------------- dtype glue
+def test_bf16_round_trip_and_rne():
+    bits = np.arange(0, 0x7F80, 7, dtype=np.uint16)          # finite positives
+    bits = np.concatenate([bits, bits | np.uint16(0x8000)])
+    v = po.bf16_to_f64(bits)
+    assert np.array_equal(po.f64_to_bf16_bits(v), bits)
+    assert np.array_equal(v.astype(np.float32), inputs.bf16_bits_to_f32(bits))
+    # halfway cases go to even; just above half goes up (also through the
+    # float32 double-rounding trap)
+    one = 1.0
+    ulp = 2.0 ** -7
+    assert po.f64_to_bf16_bits(one + ulp / 2)[()] == 0x3F80
+    assert po.f64_to_bf16_bits(one + 3 * ulp / 2)[()] == 0x3F82
+    assert po.f64_to_bf16_bits(one + ulp / 2 + 2.0 ** -40)[()] == 0x3F81
+    assert po.f64_to_bf16_bits(-(one + ulp / 2 + 2.0 ** -40))[()] == 0xBF81
+    assert po.f64_to_bf16_bits(one + ulp / 2 - 2.0 ** -40)[()] == 0x3F80
+    rng = np.random.default_rng(41)
+    vals = rng.standard_normal(2000)
+    got = po.f64_to_bf16_bits(vals)
+    for v_, b_ in zip(vals[:300], got[:300]):
+        lo = po.bf16_to_f64(np.uint16(b_ - 1))
+        mid = po.bf16_to_f64(np.uint16(b_))
+        hi = po.bf16_to_f64(np.uint16(b_ + 1))
+        assert abs(v_ - mid) <= min(abs(v_ - lo), abs(v_ - hi))
+    assert np.array_equal(inputs.f32_to_bf16_bits(vals.astype(np.float32)),
+                          po.f64_to_bf16_bits(vals.astype(np.float32).astype(np.float64)))
+
+
+def test_batch_tokens_are_independent():
+    wg, wu, wd, x = _problem(n_tok=4, seed=43)
+    dg = po.dequantize(*po.quantize_proxy(wg, 4, 128), 128)
+    du = po.dequantize(*po.quantize_proxy(wu, 4, 128), 128)
+    outs = po.forward_batch(x, 77, 100, dg, du, wg, wu, wd)
+    for t, o in enumerate(outs):
+        single = po.forward(x[t], 77, 100, dg, du, wg, wu, wd)
+        assert np.array_equal(o["y"], single["y"]) and np.array_equal(o["sel"], single["sel"])
