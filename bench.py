@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the Prox sparse-FFN hot path on B200.
+
+Metric: microseconds per Prox FFN call at 70% effective sparsity, batch 1, on
+the Qwen3-8B-shaped FFN (d_model 4096, d_ff 12288, INT4 group-128 proxy), plus
+the achieved HBM GB/s for the bytes the method must move.
+
+One *step* is one pass of the whole path over one batch of synthetic decode
+input: TOKENS consecutive single-token FFN calls, call t using weight replica
+t mod R ("layer" t mod R), so that every call streams its weights from HBM
+(R replicas x ~87 MB touched per call is far larger than the 126 MB L2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With --impl reference the CPU oracle is timed on the host cores instead.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+WORKLOAD = "qwen3_8b"
+E_PCT = 70
+PROXY = (4, 128)
+TOKENS = 512            # FFN calls per step
+REPLICAS = 24           # rotating weight sets
+METRIC = "prox_ffn_us_per_call_e70_b1"
+UNIT = "us"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="prox", choices=["prox", "reference"])
+    ap.add_argument("--tokens", type=int, default=TOKENS)
+    ap.add_argument("--replicas", type=int, default=REPLICAS)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = os.path.join("/tmp", f"prox_bench_clocks_{os.getpid()}.csv")
+
+    def start(self):
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------- CPU oracle leg
+def oracle_setup(n_tokens):
+    from oracle import prox_oracle as po
+    from paper_2607_27591_b200 import inputs
+    wl, wg, wu, wd, x = inputs.make_workload(WORKLOAD, n_tokens=n_tokens)
+    k1, k2 = wl.points[E_PCT]
+    wg32, wu32, wd32 = (inputs.bf16_bits_to_f32(a) for a in (wg, wu, wd))
+    dg = po.dequantize(*po.quantize_proxy(wg32, *PROXY), PROXY[1], np.float32)
+    du = po.dequantize(*po.quantize_proxy(wu32, *PROXY), PROXY[1], np.float32)
+    xs = po.bf16_to_f64(x)
+    return po, (k1, k2), (dg, du, wg32, wu32, wd32), xs, (wl, wg, wu, wd, x)
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def time_oracle(po, ks, mats, xs, seconds, max_tokens):
+    k1, k2 = ks
+    dg, du, wg, wu, wd = mats
+    po.forward(xs[0], k1, k2, dg, du, wg, wu, wd)          # touch everything once
+    n, t0 = 0, time.perf_counter()
+    while n < max_tokens and (n < 2 or time.perf_counter() - t0 < seconds):
+        po.forward(xs[n % len(xs)], k1, k2, dg, du, wg, wu, wd)
+        n += 1
+    dt = time.perf_counter() - t0
+    return dt / n * 1e6, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = 4
+    po, ks, mats, xs, _ = oracle_setup(per_step)
+    k1, k2 = ks
+    dg, du, wg, wu, wd = mats
+
+    def step():
+        for t in range(per_step):
+            po.forward(xs[t], k1, k2, dg, du, wg, wu, wd)
+
+    for _ in range(max(1, args.warmup)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    us = dt / (args.steps * per_step) * 1e6
+    cores = cpu_threads()
+    sample = f"{per_step} tokens per step of {WORKLOAD} e={E_PCT}% (oracle forward, proxies pre-quantized)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD} d_model=4096 d_ff=12288 e={E_PCT}% k1={k1} k2={k2} "
+                               f"int{PROXY[0]} group-{PROXY[1]} batch=1", "sample": sample},
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------ GPU leg
+def run_prox(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2607_27591_b200 import binding as pb, inputs
+
+    wl = inputs.WORKLOADS[WORKLOAD]
+    D, F = wl.d_model, wl.d_ff
+    k1, k2 = wl.points[E_PCT]
+    T, R = args.tokens, args.replicas
+
+    # replica 0 = the seeded numpy workload (also what the CPU oracle sees);
+    # the others are drawn on the device from the same distribution.
+    _, wg0, wu0, wd0, x_bits = inputs.make_workload(WORKLOAD, seed=rank, n_tokens=T)
+    as_dev = lambda b: torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).to(dev).view(torch.bfloat16)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234 + rank)
+    weights, handles = [], []
+    for r in range(R):
+        if r == 0:
+            w = (as_dev(wg0), as_dev(wu0), as_dev(wd0))
+        else:
+            w = tuple((torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * wl.w_std).to(torch.bfloat16)
+                      for shape in ((F, D), (F, D), (D, F)))
+        weights.append(w)
+        h = pb.prox_ffn_create(D, F, 8, 0, *w)
+        pb.prox_quantize_proxy(h, *PROXY)
+        handles.append(h)
+    x = as_dev(x_bits)
+    y = torch.empty(T, D, dtype=torch.bfloat16, device=dev)
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.Stream(device=dev)
+    sp = stream.cuda_stream
+
+    def enqueue_step(sptr):
+        for t in range(T):
+            pb.prox_ffn_forward(handles[t % R], x[t], 1, k1, k2, y[t], stream=sptr)
+
+    l0 = pb.prox_launch_count(handles[0])
+    graph = None
+    if not args.no_graph:
+        try:
+            with torch.cuda.stream(stream):
+                enqueue_step(sp)                       # prime (lazy module loading)
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                enqueue_step(torch.cuda.current_stream().cuda_stream)
+        except Exception as ex:                        # pragma: no cover
+            sys.stderr.write(f"graph capture failed ({ex}); timing direct launches\n")
+            graph = None
+    launches_per_call = None
+
+    def run_step():
+        if graph is not None:
+            graph.replay()
+        else:
+            enqueue_step(sp)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        c0 = sum(pb.prox_launch_count(h) for h in handles)
+        enqueue_step(sp)
+        stream.synchronize()
+        launches_per_call = (sum(pb.prox_launch_count(h) for h in handles) - c0) / T
+        for _ in range(max(3, args.warmup)):
+            run_step()
+        sync_all()
+        sampler = ClockSampler(local)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            run_step()
+        e1.record(stream)
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop()
+
+        # dominant-kernel time: per-kernel CUDA events (library hook) over one more step
+        for h in handles:
+            pb.prox_profile_enable(h, 1)
+        enqueue_step(sp)
+        stream.synchronize()
+        prof = {}
+        for h in handles:
+            for name, (n, tot_ms) in pb.prox_profile_read(h).items():
+                a = prof.setdefault(name, [0, 0.0])
+                a[0] += n; a[1] += tot_ms
+            pb.prox_profile_enable(h, 0)
+
+        # end to end through the host-buffer entry point (H2D of x, D2H of y inside the timed region)
+        xh = torch.from_numpy(np.ascontiguousarray(x_bits).view(np.int16)).view(torch.bfloat16).pin_memory()
+        yh = torch.empty(T, D, dtype=torch.bfloat16).pin_memory()
+        for t in range(min(T, 64)):
+            pb.prox_ffn_forward_host(handles[t % R], xh[t], 1, k1, k2, yh[t], stream=sp)
+        sync_all()
+        e2e_steps = max(1, min(args.steps, 5))
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for t in range(T):
+                pb.prox_ffn_forward_host(handles[t % R], xh[t], 1, k1, k2, yh[t], stream=sp)
+        sync_all()
+        e2e_s = time.perf_counter() - t0
+
+        # dense bf16 cuBLAS FFN on the same replicas (context)
+        def dense_step():
+            for t in range(T):
+                wg, wu, wd = weights[t % R]
+                g = torch.mv(wg, x[t]); u = torch.mv(wu, x[t])
+                torch.mv(wd, torch.nn.functional.silu(g) * u, out=y[t])
+        dense_us = None
+        try:
+            dense_step(); stream.synchronize()
+            dg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(dg, stream=stream):
+                dense_step()
+            for _ in range(3):
+                dg.replay()
+            stream.synchronize()
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            d0.record(stream)
+            for _ in range(5):
+                dg.replay()
+            d1.record(stream)
+            stream.synchronize()
+            dense_us = d0.elapsed_time(d1) / (5 * T) * 1e3
+        except Exception as ex:                        # pragma: no cover
+            sys.stderr.write(f"dense comparison failed: {ex}\n")
+
+    tms = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(tms[0]), float(tms[1])
+    calls = world * args.steps * T
+    us_per_call = ms * 1e3 / calls
+    e2e_us = e2e_ms * 1e3 / (world * e2e_steps * T)
+
+    s1b, gub, dnb, actb = pb.prox_algorithmic_bytes(handles[0], k1, k2)
+    bytes_call = s1b + gub + dnb + actb
+    peak, peak_kind = peaks()
+    kernel_bytes = {"input_select": 2 * D + 4 * k1, "proxy_gemv": s1b + 2 * D + 4 * k1 + 4 * F,
+                    "channel_select": 4 * F + 4 * k2, "gateup": gub + 2 * D + 8 * k2,
+                    "down": dnb + 8 * k2 + 4 * D, "finalize": 6 * D, "prox_fused": bytes_call}
+    per_kernel = {}
+    for name, (n, tot_ms) in prof.items():
+        if n:
+            us = tot_ms / n * 1e3
+            per_kernel[name] = {"us": us, "launches_per_call": n / T,
+                                "gbs": kernel_bytes.get(name, 0) / us / 1e3}
+    dom = max(per_kernel, key=lambda k: per_kernel[k]["us"] * per_kernel[k]["launches_per_call"]) if per_kernel else None
+    roof = None
+    if dom:
+        ach = per_kernel[dom]["gbs"]
+        roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s",
+                "frac": ach / peak, "peak_kind": peak_kind, "traffic": None,
+                "bytes_per_launch": kernel_bytes.get(dom)}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        po, ks, mats, xs, _ = oracle_setup(16)
+        us, n = time_oracle(po, ks, mats, xs, args.cpu_seconds, 256)
+        cpu = {"value": us, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": f"{n} tokens of the same workload (oracle forward per token, proxies pre-quantized)"}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": us_per_call, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{WORKLOAD} d_model={D} d_ff={F} e={E_PCT}% k1={k1} k2={k2} "
+                                   f"int{PROXY[0]} group-{PROXY[1]} batch=1",
+                       "calls_per_step": T, "weight_replicas": R,
+                       "l2": "inputs larger than L2: every call reads a different weight replica",
+                       "launch": "cuda graph of one step" if graph is not None else "direct launches",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single gpu"},
+            "hbm_gbs_whole_call": bytes_call / us_per_call / 1e3 * world,
+            "hbm_frac_whole_call": bytes_call / (us_per_call * world) / 1e3 / peak,
+            "algorithmic_bytes_per_call": {"stage1": s1b, "gate_up": gub, "down": dnb, "activations": actb},
+            "roofline": roof, "per_kernel": per_kernel,
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": T * D * 2, "d2h_bytes_per_step": T * D * 2},
+            "gpu_launches": int(round(launches_per_call * T * args.steps)),
+            "dense_cublas_bf16_us_per_call": dense_us,
+            "clocks": clocks,
+        }
+        print(json.dumps(out))
+    for h in handles:
+        pb.prox_ffn_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_prox(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,206 @@
+/*
+ * prox.h - C ABI of libprox: the decode-time sparse SwiGLU FFN of "Prox"
+ * (training-free FFN activation sparsity through an approximate
+ * intermediate-channel salience), written for one NVIDIA B200 (sm_100a).
+ *
+ * The path (paper Sec. 4.1 "Two-Stage Sparse Inference"):
+ *   Stage 1  proxy mask:  m_x keeps the k1 largest |x_i|; the quantized proxy
+ *            copies of W_gate and W_up are multiplied against the kept inputs
+ *            only (input sparsity Pi_in, Sec. 2.2); the proxy state
+ *            s~ = u~ (.) SiLU(g~) is ranked by magnitude and the k2 largest
+ *            channels form the mask m_s shared by all three projections.
+ *   Stage 2  exact sparse compute:  for the channels in m_s, gate and up are
+ *            recomputed with the original bf16 weights and the dense x
+ *            (output sparsity Pi_out), s = u (.) SiLU(g), and the down
+ *            projection sums s_j * W_down[j,:] over those channels only.
+ *
+ * Selection rule: the paper's main rule is a calibrated layer threshold
+ * (indicator |z| >= tau); this library implements the per-token top-k rule of
+ * the appendix "Threshold-Based Selection and Token-Adaptive Computation"
+ * (exactly k entries, ties go to the lower index) and, as a variant, the
+ * threshold rule with caller-supplied tau (prox_*_threshold entry points).
+ *
+ * Conventions for every call
+ *   - "dev" pointers are CUDA device pointers on the current device, "host"
+ *     pointers are ordinary host memory.  Nothing here takes a framework type.
+ *   - Matrices are row-major with the nn.Linear orientation:
+ *       W_gate, W_up : bf16 [d_ff, d_model]   row j = weights of channel j
+ *       W_down       : bf16 [d_model, d_ff]
+ *     (the paper writes W_up, W_gate in R^{d_model x d_ff}, W_down in
+ *     R^{d_ff x d_model}; these are the transposes, Sec. 2.1).
+ *   - x is bf16 [B, d_model]; y is [B, d_model] in the handle's out_dtype.
+ *     Each of the B tokens gets its own masks (the paper covers B = 1 only).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
+ *     is enqueued on it and the call returns without synchronising unless the
+ *     call's comment says otherwise.  A handle must not be used from two
+ *     streams at once: its scratch buffers are shared by all calls.
+ *   - Every call validates its arguments on the host and returns a status;
+ *     nothing throws or aborts across this boundary.  Inputs are assumed
+ *     finite; NaN/Inf in x or the weights give unspecified masks.
+ *   - Caller-owned memory: x, y, sel, scores and the original weights.
+ *     w_gate and w_up are BORROWED for the handle's whole life (Stage 2 reads
+ *     them in place); w_down is read only by prox_quantize_proxy.  The handle
+ *     owns the packed proxies, their scales, the channel-major copy of W_down
+ *     and all scratch.
+ */
+#ifndef PROX_H_
+#define PROX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct prox_ffn prox_ffn_t;
+
+typedef enum {
+  PROX_OK = 0,
+  PROX_ERR_INVALID_ARG = 1,   /* null pointer, size out of range, misaligned pointer */
+  PROX_ERR_UNSUPPORTED = 2,   /* shape / bits / group_size this build does not handle */
+  PROX_ERR_NOT_QUANTIZED = 3, /* Stage 1 asked for before prox_quantize_proxy */
+  PROX_ERR_CUDA = 4,          /* a CUDA runtime call failed (incl. no device) */
+  PROX_ERR_OOM = 5,           /* device or host allocation failed */
+  PROX_ERR_TIMEOUT = 6,       /* a bounded device-side wait gave up */
+  PROX_ERR_IO = 7             /* file could not be read / written / parsed */
+} prox_status_t;
+
+typedef struct {
+  int32_t d_model;   /* D: multiple of 128, 128..16384 */
+  int32_t d_ff;      /* F: multiple of 64,  64..65536  */
+  int32_t max_batch; /* 1..8 tokens per call */
+  int32_t out_dtype; /* 0 = bf16, 1 = fp32 */
+} prox_ffn_config_t;
+
+/* Create a handle over caller-owned dev bf16 weights (Sec. 2.1 for the shapes).
+ * Pointers must be 16-byte aligned.  Allocates scratch; copies nothing.
+ * Errors: INVALID_ARG, UNSUPPORTED (shape), CUDA, OOM. */
+prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate_dev,
+                              const void* w_up_dev, const void* w_down_dev,
+                              void* stream, prox_ffn_t** out);
+
+/* Offline packer (Sec. 4.3: "symmetric per-row INT4 quantization of the
+ * original W_up and W_gate ... keeping the compact proxies resident in GPU
+ * memory").  For every channel j and every group of `group_size` consecutive
+ * input indices (0 = the whole row, the paper's per-row case):
+ *     scale = fp16(max|w| / qmax),  qmax = 2^(bits-1)-1
+ *     q     = clamp(rint(w / scale), -qmax, qmax)      (fp32, ties to even)
+ * Proxies are stored input-major (all channels of one input coordinate are
+ * contiguous, gate and up interleaved) so that Stage 1's input sparsity skips
+ * whole rows of bytes.  Also writes the channel-major copy of W_down
+ * ([d_ff, d_model], Sec. 3.1: y = sum_j s_j W_down[j,:]) so that the masked
+ * down projection reads one contiguous row per kept channel.
+ * bits in {4, 8}; group_size in {0, 128}.  May be called again to re-pack.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA, OOM. */
+prox_status_t prox_quantize_proxy(prox_ffn_t* h, int bits, int group_size, void* stream);
+
+/* Stage 1 (Sec. 4.1, "lightweight proxy construction"), top-k rule.
+ *   x          dev bf16 [B, D]
+ *   k1         kept inputs per token, 1..D   (k1 = D keeps every input)
+ *   k2         kept channels per token, 1..F
+ *   sel        dev int32 [B, k2] out: kept channel ids, ascending, per token
+ *   scores     dev fp32 [B, F] out or NULL: |u~_j * SiLU(g~_j)|
+ * Errors: INVALID_ARG, NOT_QUANTIZED, CUDA. */
+prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x_dev, int B, int k1, int k2,
+                               int32_t* sel_dev, float* scores_dev_or_null, void* stream);
+
+/* Stage 2 (Sec. 4.1, "exact sparse computation") for a given mask.
+ *   sel        dev int32 [B, k2]: channel ids per token, each in [0, F),
+ *              ascending and unique within a token (as Stage 1 writes them)
+ *   y          dev [B, D] out, out_dtype
+ * Out-of-range ids are skipped and recorded (see prox_last_device_status).
+ * Needs the channel-major W_down, i.e. prox_quantize_proxy must have run.
+ * Errors: INVALID_ARG, NOT_QUANTIZED, CUDA. */
+prox_status_t prox_stage2_ffn(prox_ffn_t* h, const void* x_dev, int B, const int32_t* sel_dev,
+                              int k2, void* y_dev, void* stream);
+
+/* Stage 1 then Stage 2 on one stream; the mask stays on the device. */
+prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x_dev, int B, int k1, int k2,
+                               void* y_dev, void* stream);
+
+/* Same as prox_ffn_forward with HOST buffers: copies x (host bf16 [B, D]) to
+ * the device, runs the path, copies y back and synchronises the stream before
+ * returning.  Pinned host memory makes the copies asynchronous w.r.t. other
+ * streams; pageable memory also works. */
+prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, int k1, int k2,
+                                    void* y_host, void* stream);
+
+/* Threshold variant of the two indicators of Sec. 4.1:
+ *   [m_x]_i = 1[|x_i| >= tau_x],  [m_s]_j = 1[|s~_j| >= tau_s].
+ * The number of kept entries varies per token.
+ *   count_dev  dev int32 [B] out: kept channels per token
+ *   sel        dev int32 [B, F] out: first count[b] entries of row b are valid
+ * prox_stage2_ffn_var consumes that layout (row stride F). */
+prox_status_t prox_stage1_mask_threshold(prox_ffn_t* h, const void* x_dev, int B, float tau_x,
+                                         float tau_s, int32_t* sel_dev, int32_t* count_dev,
+                                         float* scores_dev_or_null, void* stream);
+prox_status_t prox_stage2_ffn_var(prox_ffn_t* h, const void* x_dev, int B, const int32_t* sel_dev,
+                                  const int32_t* count_dev, void* y_dev, void* stream);
+prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x_dev, int B, float tau_x,
+                                         float tau_s, void* y_dev, void* stream);
+
+/* Runtime mask counts accumulated by the threshold entry points since the last
+ * reset (appendix "Threshold Calibration and Runtime Sparsity":
+ * e^ = s2^ - 2 alpha (1 - s1^) / 3).  Host-synchronous.  Any pointer may be NULL. */
+prox_status_t prox_runtime_sparsity(prox_ffn_t* h, double alpha, int64_t* tokens,
+                                    double* s1_hat, double* s2_hat, double* e_hat, int reset);
+
+/* Budget helper (Sec. 4.2): s2 = s_ref, s1 from e = s2 - 2 alpha (1 - s1) / 3;
+ * if s1 leaves [s1_min, s1_max] it is clamped and s2 re-solved.  Host only. */
+prox_status_t prox_allocate_budget(double e, double alpha, double s_ref, double s1_min,
+                                   double s1_max, double* s1, double* s2);
+
+/* k = clamp(floor((1 - s) * dim + 0.5), 1, dim).  Host only. */
+prox_status_t prox_sparsity_to_k(double s, int dim, int* k);
+
+/* Test hook: unpack the stored proxy of W_gate (which = 0) or W_up (1) into
+ * host q int8 [F, D] and host scale fp32 [F, D/group] (group = D if per-row).
+ * Synchronises.  Errors: INVALID_ARG, NOT_QUANTIZED, CUDA, OOM. */
+prox_status_t prox_proxy_export(prox_ffn_t* h, int which, int8_t* q_host, float* scale_host);
+
+/* Test hook: the Stage-1 input mask alone.  idx dev int32 [B, k1], ascending. */
+prox_status_t prox_input_topk(prox_ffn_t* h, const void* x_dev, int B, int k1,
+                              int32_t* idx_dev, void* stream);
+
+/* Offline packer output: write / read the packed proxies, scales and the
+ * channel-major W_down of a quantized handle.  prox_pack_load needs a handle
+ * created over the same weights and shape; it replaces prox_quantize_proxy.
+ * Both synchronise.  Errors: INVALID_ARG, NOT_QUANTIZED, IO, CUDA, OOM. */
+prox_status_t prox_pack_save(prox_ffn_t* h, const char* path);
+prox_status_t prox_pack_load(prox_ffn_t* h, const char* path, void* stream);
+
+/* Bytes the method must move for one call at these budgets (B = 1 layout,
+ * `rows_in` kept input rows and `rows_ch` kept channel rows actually read):
+ * proxy rows + scales + gate/up rows + down rows + activations.  Host only. */
+prox_status_t prox_algorithmic_bytes(const prox_ffn_t* h, int rows_in, int rows_ch,
+                                     int64_t* stage1, int64_t* gate_up, int64_t* down,
+                                     int64_t* activations);
+
+/* Device-side diagnostics: 0 if no kernel recorded a problem since the last
+ * read; otherwise a bit set (1 = channel id out of range skipped, 2 = input id
+ * out of range skipped, 4 = bounded wait expired).  Reading clears it.
+ * Synchronises the given stream. */
+prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream);
+
+/* Per-kernel timing hook for benchmarks.  While enabled, every kernel launched
+ * through the handle is bracketed by CUDA events on the call's stream (this
+ * adds event records to the stream and must not be on during stream capture).
+ * prox_profile_read synchronises those events, adds up launches and
+ * milliseconds per kernel kind into counts[PROX_NUM_KERNEL_KINDS] and
+ * ms[PROX_NUM_KERNEL_KINDS] (host arrays), and forgets them.  Kinds, in order:
+ * input_select, proxy_gemv, channel_select, gateup, down, finalize, fused. */
+#define PROX_NUM_KERNEL_KINDS 7
+prox_status_t prox_profile_enable(prox_ffn_t* h, int on);
+prox_status_t prox_profile_read(prox_ffn_t* h, int64_t* counts_host, double* ms_host);
+
+/* Number of kernels this library launched through the handle so far. */
+prox_status_t prox_launch_count(const prox_ffn_t* h, int64_t* launches);
+
+void prox_ffn_destroy(prox_ffn_t* h);
+const char* prox_status_string(prox_status_t s);
+const char* prox_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROX_H_ */

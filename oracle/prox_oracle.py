@@ -119,13 +119,15 @@ def quantize_proxy(w, bits: int, group_size: int):
     return q.reshape(d_ff, d_model).astype(np.int8), scale
 
 
-def dequantize(q, scale, group_size: int) -> np.ndarray:
-    """deq[j, i] = q[j, i] * scale[j, i // group]  in float64."""
+def dequantize(q, scale, group_size: int, dtype=np.float64) -> np.ndarray:
+    """deq[j, i] = q[j, i] * scale[j, i // group].  The product of an 8-bit
+    integer and an fp16 value has at most 19 significant bits, so it is exact in
+    float32 as well as in float64 (`dtype` only chooses the storage)."""
     q = np.asarray(q)
     d_ff, d_model = q.shape
     g = d_model if group_size == 0 else group_size
-    s = np.asarray(scale, dtype=np.float64).reshape(d_ff, d_model // g)
-    return (q.astype(np.float64).reshape(d_ff, d_model // g, g) * s[:, :, None]).reshape(d_ff, d_model)
+    s = np.asarray(scale).astype(dtype).reshape(d_ff, d_model // g)
+    return (q.astype(dtype).reshape(d_ff, d_model // g, g) * s[:, :, None]).reshape(d_ff, d_model)
 
 
 # ------------------------------------------------------------ Stage 1 masks
@@ -151,7 +153,7 @@ def input_sparse_projection(x, idx, w) -> np.ndarray:
     input coordinates contribute.  `w` is stored [d_out, d_in]."""
     x = np.asarray(x, dtype=np.float64)
     idx = np.asarray(idx, dtype=np.int64)
-    return np.asarray(w, dtype=np.float64)[:, idx] @ x[idx]
+    return np.asarray(w)[:, idx].astype(np.float64) @ x[idx]
 
 
 def proxy_scores(x, idx_x, deq_gate, deq_up) -> np.ndarray:
@@ -185,10 +187,10 @@ def stage2(x, sel, w_gate, w_up, w_down):
     The dense x and the original weights are used.  Returns (y, s_sp)."""
     x = np.asarray(x, dtype=np.float64)
     sel = np.asarray(sel, dtype=np.int64)
-    u_sp = np.asarray(w_up, dtype=np.float64)[sel, :] @ x
-    h_sp = silu(np.asarray(w_gate, dtype=np.float64)[sel, :] @ x)
+    u_sp = np.asarray(w_up)[sel, :].astype(np.float64) @ x
+    h_sp = silu(np.asarray(w_gate)[sel, :].astype(np.float64) @ x)
     s_sp = u_sp * h_sp
-    y = np.asarray(w_down, dtype=np.float64)[:, sel] @ s_sp
+    y = np.asarray(w_down)[:, sel].astype(np.float64) @ s_sp
     return y, s_sp
 
 

@@ -1,0 +1,230 @@
+"""Thin ctypes binding over libprox.so (declared in include/prox.h).
+
+Argument marshalling only: every function here has the name of the C entry
+point it forwards to, takes raw device pointers (Python ints, e.g.
+``tensor.data_ptr()``) or objects exposing ``data_ptr()``, and raises
+``ProxError`` when the library returns a non-zero status.  No step of the
+path is computed in Python and there is no fallback: if the shared library
+is missing the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libprox.so")
+
+STATUS_NAMES = {
+    0: "PROX_OK", 1: "PROX_ERR_INVALID_ARG", 2: "PROX_ERR_UNSUPPORTED", 3: "PROX_ERR_NOT_QUANTIZED",
+    4: "PROX_ERR_CUDA", 5: "PROX_ERR_OOM", 6: "PROX_ERR_TIMEOUT", 7: "PROX_ERR_IO",
+}
+
+
+class ProxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({prox_status_string(status)})")
+
+
+class ProxFFNConfig(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("d_ff", C.c_int32), ("max_batch", C.c_int32),
+                ("out_dtype", C.c_int32)]
+
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2607_27591_b200.build` "
+        "(needs nvcc). There is no fallback implementation.")
+_lib = C.CDLL(_LIB_PATH)
+
+_vp, _i, _f, _d = C.c_void_p, C.c_int, C.c_float, C.c_double
+_SIGS = {
+    "prox_ffn_create": [C.POINTER(ProxFFNConfig), _vp, _vp, _vp, _vp, C.POINTER(_vp)],
+    "prox_quantize_proxy": [_vp, _i, _i, _vp],
+    "prox_stage1_mask": [_vp, _vp, _i, _i, _i, _vp, _vp, _vp],
+    "prox_stage2_ffn": [_vp, _vp, _i, _vp, _i, _vp, _vp],
+    "prox_ffn_forward": [_vp, _vp, _i, _i, _i, _vp, _vp],
+    "prox_ffn_forward_host": [_vp, _vp, _i, _i, _i, _vp, _vp],
+    "prox_stage1_mask_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp, _vp, _vp],
+    "prox_stage2_ffn_var": [_vp, _vp, _i, _vp, _vp, _vp, _vp],
+    "prox_ffn_forward_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp],
+    "prox_runtime_sparsity": [_vp, _d, C.POINTER(C.c_int64), C.POINTER(_d), C.POINTER(_d), C.POINTER(_d), _i],
+    "prox_allocate_budget": [_d, _d, _d, _d, _d, C.POINTER(_d), C.POINTER(_d)],
+    "prox_sparsity_to_k": [_d, _i, C.POINTER(_i)],
+    "prox_proxy_export": [_vp, _i, _vp, _vp],
+    "prox_input_topk": [_vp, _vp, _i, _i, _vp, _vp],
+    "prox_pack_save": [_vp, C.c_char_p],
+    "prox_pack_load": [_vp, C.c_char_p, _vp],
+    "prox_algorithmic_bytes": [_vp, _i, _i, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                               C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
+    "prox_last_device_status": [_vp, C.POINTER(C.c_int32), _vp],
+    "prox_launch_count": [_vp, C.POINTER(C.c_int64)],
+    "prox_profile_enable": [_vp, _i],
+    "prox_profile_read": [_vp, C.POINTER(C.c_int64), C.POINTER(_d)],
+}
+for _name, _args in _SIGS.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes = _args
+    _fn.restype = C.c_int
+_lib.prox_ffn_destroy.argtypes = [_vp]
+_lib.prox_ffn_destroy.restype = None
+_lib.prox_status_string.argtypes = [C.c_int]
+_lib.prox_status_string.restype = C.c_char_p
+_lib.prox_version.argtypes = []
+_lib.prox_version.restype = C.c_char_p
+
+EXPORTED = tuple(_SIGS) + ("prox_ffn_destroy", "prox_status_string", "prox_version")
+
+
+def _ptr(obj) -> Optional[int]:
+    """Raw address of a device/host buffer: int, None, or anything with data_ptr()."""
+    if obj is None:
+        return None
+    if isinstance(obj, int):
+        return obj
+    if hasattr(obj, "data_ptr"):
+        return obj.data_ptr()
+    if hasattr(obj, "ctypes"):                       # numpy array (host memory)
+        return obj.ctypes.data
+    raise TypeError(f"cannot take the address of {type(obj)}")
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise ProxError(status, where)
+
+
+def prox_status_string(status: int) -> str:
+    return _lib.prox_status_string(int(status)).decode()
+
+
+def prox_version() -> str:
+    return _lib.prox_version().decode()
+
+
+def prox_ffn_create(d_model: int, d_ff: int, max_batch: int, out_dtype: int, w_gate, w_up, w_down,
+                    stream=None) -> int:
+    cfg = ProxFFNConfig(d_model, d_ff, max_batch, out_dtype)
+    out = _vp()
+    _check(_lib.prox_ffn_create(C.byref(cfg), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(stream),
+                                C.byref(out)), "prox_ffn_create")
+    return out.value
+
+
+def prox_ffn_destroy(handle: int) -> None:
+    _lib.prox_ffn_destroy(handle)
+
+
+def prox_quantize_proxy(handle: int, bits: int, group_size: int, stream=None) -> None:
+    _check(_lib.prox_quantize_proxy(handle, bits, group_size, _ptr(stream)), "prox_quantize_proxy")
+
+
+def prox_stage1_mask(handle: int, x, B: int, k1: int, k2: int, sel, scores=None, stream=None) -> None:
+    _check(_lib.prox_stage1_mask(handle, _ptr(x), B, k1, k2, _ptr(sel), _ptr(scores), _ptr(stream)),
+           "prox_stage1_mask")
+
+
+def prox_stage2_ffn(handle: int, x, B: int, sel, k2: int, y, stream=None) -> None:
+    _check(_lib.prox_stage2_ffn(handle, _ptr(x), B, _ptr(sel), k2, _ptr(y), _ptr(stream)), "prox_stage2_ffn")
+
+
+def prox_ffn_forward(handle: int, x, B: int, k1: int, k2: int, y, stream=None) -> None:
+    _check(_lib.prox_ffn_forward(handle, _ptr(x), B, k1, k2, _ptr(y), _ptr(stream)), "prox_ffn_forward")
+
+
+def prox_ffn_forward_host(handle: int, x_host, B: int, k1: int, k2: int, y_host, stream=None) -> None:
+    _check(_lib.prox_ffn_forward_host(handle, _ptr(x_host), B, k1, k2, _ptr(y_host), _ptr(stream)),
+           "prox_ffn_forward_host")
+
+
+def prox_stage1_mask_threshold(handle: int, x, B: int, tau_x: float, tau_s: float, sel, count,
+                               scores=None, stream=None) -> None:
+    _check(_lib.prox_stage1_mask_threshold(handle, _ptr(x), B, tau_x, tau_s, _ptr(sel), _ptr(count),
+                                           _ptr(scores), _ptr(stream)), "prox_stage1_mask_threshold")
+
+
+def prox_stage2_ffn_var(handle: int, x, B: int, sel, count, y, stream=None) -> None:
+    _check(_lib.prox_stage2_ffn_var(handle, _ptr(x), B, _ptr(sel), _ptr(count), _ptr(y), _ptr(stream)),
+           "prox_stage2_ffn_var")
+
+
+def prox_ffn_forward_threshold(handle: int, x, B: int, tau_x: float, tau_s: float, y, stream=None) -> None:
+    _check(_lib.prox_ffn_forward_threshold(handle, _ptr(x), B, tau_x, tau_s, _ptr(y), _ptr(stream)),
+           "prox_ffn_forward_threshold")
+
+
+def prox_runtime_sparsity(handle: int, alpha: float = 1.0 / 3.0, reset: bool = False):
+    tok, s1, s2, e = C.c_int64(), _d(), _d(), _d()
+    _check(_lib.prox_runtime_sparsity(handle, alpha, C.byref(tok), C.byref(s1), C.byref(s2), C.byref(e),
+                                      int(reset)), "prox_runtime_sparsity")
+    return tok.value, s1.value, s2.value, e.value
+
+
+def prox_allocate_budget(e: float, alpha: float = 1.0 / 3.0, s_ref: float = 0.7, s1_min: float = 0.0,
+                         s1_max: float = 0.7) -> Tuple[float, float]:
+    s1, s2 = _d(), _d()
+    _check(_lib.prox_allocate_budget(e, alpha, s_ref, s1_min, s1_max, C.byref(s1), C.byref(s2)),
+           "prox_allocate_budget")
+    return s1.value, s2.value
+
+
+def prox_sparsity_to_k(s: float, dim: int) -> int:
+    k = _i()
+    _check(_lib.prox_sparsity_to_k(s, dim, C.byref(k)), "prox_sparsity_to_k")
+    return k.value
+
+
+def prox_proxy_export(handle: int, which: int, q_host, scale_host) -> None:
+    _check(_lib.prox_proxy_export(handle, which, _ptr(q_host), _ptr(scale_host)), "prox_proxy_export")
+
+
+def prox_input_topk(handle: int, x, B: int, k1: int, idx, stream=None) -> None:
+    _check(_lib.prox_input_topk(handle, _ptr(x), B, k1, _ptr(idx), _ptr(stream)), "prox_input_topk")
+
+
+def prox_pack_save(handle: int, path: str) -> None:
+    _check(_lib.prox_pack_save(handle, os.fsencode(path)), "prox_pack_save")
+
+
+def prox_pack_load(handle: int, path: str, stream=None) -> None:
+    _check(_lib.prox_pack_load(handle, os.fsencode(path), _ptr(stream)), "prox_pack_load")
+
+
+def prox_algorithmic_bytes(handle: int, rows_in: int, rows_ch: int):
+    a, b, c, d = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64()
+    _check(_lib.prox_algorithmic_bytes(handle, rows_in, rows_ch, C.byref(a), C.byref(b), C.byref(c),
+                                       C.byref(d)), "prox_algorithmic_bytes")
+    return a.value, b.value, c.value, d.value
+
+
+def prox_last_device_status(handle: int, stream=None) -> int:
+    code = C.c_int32()
+    _check(_lib.prox_last_device_status(handle, C.byref(code), _ptr(stream)), "prox_last_device_status")
+    return code.value
+
+
+def prox_launch_count(handle: int) -> int:
+    n = C.c_int64()
+    _check(_lib.prox_launch_count(handle, C.byref(n)), "prox_launch_count")
+    return n.value
+
+
+KERNEL_KINDS = ("input_select", "proxy_gemv", "channel_select", "gateup", "down", "finalize", "prox_fused")
+
+
+def prox_profile_enable(handle: int, on: int) -> None:
+    _check(_lib.prox_profile_enable(handle, int(on)), "prox_profile_enable")
+
+
+def prox_profile_read(handle: int):
+    """{kernel kind: (launches, total milliseconds)} since the last read."""
+    n = (C.c_int64 * len(KERNEL_KINDS))()
+    ms = (_d * len(KERNEL_KINDS))()
+    _check(_lib.prox_profile_read(handle, n, ms), "prox_profile_read")
+    return {k: (n[i], ms[i]) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def raw(name: str):
+    """The raw ctypes function (returns the status instead of raising); for tests of error paths."""
+    return getattr(_lib, name)

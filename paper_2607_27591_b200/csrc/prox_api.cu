@@ -1,0 +1,659 @@
+// Host side of libprox: argument validation, memory ownership, launches.
+// Declarations and per-call documentation live in include/prox.h.
+#include "prox.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "prox_kernels.cuh"
+
+using namespace prox;
+
+enum KernelKind { kKInput = 0, kKProxy, kKChannel, kKGateUp, kKDown, kKFinalize, kKFused };
+struct ProfRec { int kind; cudaEvent_t a, b; };
+
+struct prox_ffn {
+  prox_ffn_config_t cfg;
+  const uint16_t* wg;
+  const uint16_t* wu;
+  const uint16_t* wd;
+  int device;
+  int sm_count;
+  // packed state (owned)
+  int bits, group;          // group = actual group length (D when per-row)
+  bool quantized;
+  uint8_t* P;               // [D][F*bits/4]
+  size_t p_bytes;
+  __half* S;                // [ngroups][nchunks][2][CH]
+  size_t s_count;
+  float* s_plain;           // [2][F][ngroups] fp32 copy of the scales
+  uint16_t* wdt;            // [F][D]
+  // scratch (owned)
+  int* idx_x;               // [maxB][D]
+  int* cnt_x;               // [maxB]
+  float* part;              // split-K partial sums
+  size_t part_floats;
+  unsigned* ticket;         // [maxB][nstrips_max]
+  float* scores;            // [maxB][F]
+  int* sel;                 // [maxB][F]
+  int* cnt_s;               // [maxB]
+  float* hbuf;              // [maxB][F]
+  float* yacc;              // [maxB][D]
+  int* dev_status;
+  unsigned long long* counters;  // [0] tokens, [1] kept inputs, [2] kept channels
+  void* x_stage;            // device staging for the host-buffer entry point
+  void* y_stage;
+  int64_t launches;
+  bool profiling;
+  std::vector<ProfRec>* prof;
+};
+
+namespace {
+
+#define CK(expr)                                   \
+  do {                                             \
+    cudaError_t e_ = (expr);                       \
+    if (e_ != cudaSuccess) return map_cuda(e_);    \
+  } while (0)
+
+prox_status_t map_cuda(cudaError_t e) {
+  if (e == cudaErrorMemoryAllocation) return PROX_ERR_OOM;
+  return PROX_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int ch_per_chunk(int bits) { return bits == 4 ? 16 : 8; }
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t count) {
+  *p = nullptr;
+  return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T) > 0 ? count * sizeof(T) : 16);
+}
+
+void free_packed(prox_ffn* h) {
+  cudaFree(h->P); cudaFree(h->S); cudaFree(h->s_plain); cudaFree(h->wdt);
+  h->P = nullptr; h->S = nullptr; h->s_plain = nullptr; h->wdt = nullptr;
+  h->quantized = false;
+}
+
+prox_status_t alloc_packed(prox_ffn* h, int bits, int group_len) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  free_packed(h);
+  h->bits = bits;
+  h->group = group_len;
+  const int CH = ch_per_chunk(bits);
+  const int nchunks = F / CH, ngroups = D / group_len;
+  h->p_bytes = (size_t)D * nchunks * 16;
+  h->s_count = (size_t)ngroups * nchunks * 2 * CH;
+  CK(dev_alloc(&h->P, h->p_bytes));
+  CK(dev_alloc(&h->S, h->s_count));
+  CK(dev_alloc(&h->s_plain, (size_t)2 * F * ngroups));
+  CK(dev_alloc(&h->wdt, (size_t)F * D));
+  return PROX_OK;
+}
+
+int nstrips_for(int F, int bits) {
+  const int per_strip = 32 * ch_per_chunk(bits);
+  return (F + per_strip - 1) / per_strip;
+}
+
+int ksplit_for(const prox_ffn* h, int B, int n_rows) {
+  const int ns = nstrips_for(h->cfg.d_ff, h->bits);
+  int target = 2 * h->sm_count;
+  int ks = (target + ns * B - 1) / (ns * B);
+  const int by_rows = n_rows / 32 > 1 ? n_rows / 32 : 1;   // keep >= 4 rows per warp
+  if (ks > by_rows) ks = by_rows;
+  if (ks > 32) ks = 32;
+  if (ks < 1) ks = 1;
+  return ks;
+}
+
+prox_status_t check_common(const prox_ffn* h, const void* x, int B) {
+  if (!h || !x) return PROX_ERR_INVALID_ARG;
+  if (B < 1 || B > h->cfg.max_batch) return PROX_ERR_INVALID_ARG;
+  if (!aligned16(x)) return PROX_ERR_INVALID_ARG;
+  return PROX_OK;
+}
+
+// Brackets one launch with events when the handle's timing hook is on.
+struct LaunchScope {
+  prox_ffn* h; cudaStream_t st; ProfRec rec; bool on;
+  LaunchScope(prox_ffn* h_, int kind, cudaStream_t st_) : h(h_), st(st_), on(h_->profiling) {
+    rec.kind = kind; rec.a = rec.b = nullptr;
+    if (on) {
+      if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) { on = false; return; }
+      cudaEventRecord(rec.a, st);
+    }
+  }
+  ~LaunchScope() {
+    h->launches++;
+    if (on) { cudaEventRecord(rec.b, st); h->prof->push_back(rec); }
+  }
+};
+
+// ---- launches ---------------------------------------------------------------
+prox_status_t launch_input_select(prox_ffn* h, const void* x, int B, int k1, float tau, int use_tau,
+                                  int* idx, int stride, int* cnt, cudaStream_t st) {
+  {
+    LaunchScope ls(h, kKInput, st);
+    input_select_kernel<<<B, kSelThreads, 0, st>>>(static_cast<const uint16_t*>(x), h->cfg.d_model, k1,
+                                                   tau, use_tau, idx, stride, cnt);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+prox_status_t launch_proxy(prox_ffn* h, const void* x, int B, const int* idx, int stride,
+                           const int* cnt, int k1, float* scores, cudaStream_t st) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  const int ns = nstrips_for(F, h->bits);
+  const int ks = ksplit_for(h, B, k1);
+  const int gshift = (h->group == D) ? 31 : 7;
+  dim3 grid(ns, ks, B);
+  const size_t need = (size_t)B * ks * ns * 2 * ch_per_chunk(h->bits) * 32;
+  if (ks > 1 && need > h->part_floats) return PROX_ERR_UNSUPPORTED;
+  LaunchScope ls(h, kKProxy, st);
+  if (h->bits == 4) {
+    const size_t smem = (size_t)kProxyWarps * ProxyFmt<4>::NACC * 32 * sizeof(float);
+    proxy_gemv_kernel<4><<<grid, kProxyThreads, smem, st>>>(
+        h->P, h->S, static_cast<const uint16_t*>(x), idx, stride, cnt, k1, D, F, gshift, h->part,
+        h->ticket, scores, h->dev_status);
+  } else {
+    const size_t smem = (size_t)kProxyWarps * ProxyFmt<8>::NACC * 32 * sizeof(float);
+    proxy_gemv_kernel<8><<<grid, kProxyThreads, smem, st>>>(
+        h->P, h->S, static_cast<const uint16_t*>(x), idx, stride, cnt, k1, D, F, gshift, h->part,
+        h->ticket, scores, h->dev_status);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+prox_status_t launch_channel_select(prox_ffn* h, const float* scores, int B, int k2, float tau,
+                                    int use_tau, int* sel, int stride, int* cnt, cudaStream_t st) {
+  {
+    LaunchScope ls(h, kKChannel, st);
+    channel_select_kernel<<<B, kSelThreads, 0, st>>>(scores, h->cfg.d_ff, k2, tau, use_tau, sel, stride, cnt);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, int stride,
+                            const int* cnt, int k2, void* y, cudaStream_t st) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  const int wpb = kGateUpThreads / 32;
+  dim3 g1((k2 + wpb - 1) / wpb, B);
+  {
+    LaunchScope ls(h, kKGateUp, st);
+    gateup_kernel<<<g1, kGateUpThreads, (size_t)D * 2, st>>>(
+        h->wg, h->wu, static_cast<const uint16_t*>(x), sel, stride, cnt, k2, D, F, h->hbuf, F,
+        h->dev_status);
+  }
+  CK(cudaGetLastError());
+  const int dtiles = (D + kDownThreads * 8 - 1) / (kDownThreads * 8);
+  int nsplit = (2 * h->sm_count + dtiles * B - 1) / (dtiles * B);
+  if (nsplit > k2) nsplit = k2;
+  if (nsplit < 1) nsplit = 1;
+  dim3 g2(dtiles, nsplit, B);
+  {
+    LaunchScope ls(h, kKDown, st);
+    down_kernel<<<g2, kDownThreads, 0, st>>>(h->wdt, h->hbuf, F, sel, stride, cnt, k2, D, F, h->yacc);
+  }
+  CK(cudaGetLastError());
+  const int n = B * D;
+  {
+    LaunchScope ls(h, kKFinalize, st);
+    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, y, n, h->cfg.out_dtype);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+}  // namespace
+
+// ============================================================================
+extern "C" {
+
+prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, const void* w_up,
+                              const void* w_down, void* stream, prox_ffn_t** out) {
+  (void)stream;
+  if (!out) return PROX_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || !w_gate || !w_up || !w_down) return PROX_ERR_INVALID_ARG;
+  if (!aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down)) return PROX_ERR_INVALID_ARG;
+  if (cfg->max_batch < 1 || cfg->max_batch > kMaxBatch) return PROX_ERR_INVALID_ARG;
+  if (cfg->out_dtype != 0 && cfg->out_dtype != 1) return PROX_ERR_INVALID_ARG;
+  if (cfg->d_model <= 0 || cfg->d_ff <= 0) return PROX_ERR_INVALID_ARG;
+  if (cfg->d_model % 128 || cfg->d_model > 16384) return PROX_ERR_UNSUPPORTED;
+  if (cfg->d_ff % 64 || cfg->d_ff > 65536) return PROX_ERR_UNSUPPORTED;
+
+  prox_ffn* h = new (std::nothrow) prox_ffn();
+  if (!h) return PROX_ERR_OOM;
+  std::memset(h, 0, sizeof(*h));
+  h->prof = new (std::nothrow) std::vector<ProfRec>();
+  if (!h->prof) { delete h; return PROX_ERR_OOM; }
+  h->cfg = *cfg;
+  h->wg = static_cast<const uint16_t*>(w_gate);
+  h->wu = static_cast<const uint16_t*>(w_up);
+  h->wd = static_cast<const uint16_t*>(w_down);
+  cudaError_t e = cudaGetDevice(&h->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+  if (e != cudaSuccess) { delete h; return PROX_ERR_CUDA; }
+
+  const int D = cfg->d_model, F = cfg->d_ff, MB = cfg->max_batch;
+  const int ns_max = nstrips_for(F, 8);            // 8-bit strips are narrower -> more of them
+  h->part_floats = ((size_t)2 * h->sm_count + (size_t)MB * ns_max + 64) * 1024;
+  prox_status_t st = PROX_OK;
+  auto A = [&](cudaError_t er) { if (er != cudaSuccess && st == PROX_OK) st = map_cuda(er); };
+  A(dev_alloc(&h->idx_x, (size_t)MB * D));
+  A(dev_alloc(&h->cnt_x, (size_t)MB));
+  A(dev_alloc(&h->part, h->part_floats));
+  A(dev_alloc(&h->ticket, (size_t)MB * ns_max));
+  A(dev_alloc(&h->scores, (size_t)MB * F));
+  A(dev_alloc(&h->sel, (size_t)MB * F));
+  A(dev_alloc(&h->cnt_s, (size_t)MB));
+  A(dev_alloc(&h->hbuf, (size_t)MB * F));
+  A(dev_alloc(&h->yacc, (size_t)MB * D));
+  A(dev_alloc(&h->dev_status, (size_t)1));
+  A(dev_alloc(&h->counters, (size_t)4));
+  A(dev_alloc(reinterpret_cast<uint16_t**>(&h->x_stage), (size_t)MB * D));
+  A(dev_alloc(reinterpret_cast<float**>(&h->y_stage), (size_t)MB * D));
+  if (st == PROX_OK) {
+    A(cudaMemset(h->ticket, 0, (size_t)MB * ns_max * sizeof(unsigned)));
+    A(cudaMemset(h->yacc, 0, (size_t)MB * D * sizeof(float)));
+    A(cudaMemset(h->dev_status, 0, sizeof(int)));
+    A(cudaMemset(h->counters, 0, 4 * sizeof(unsigned long long)));
+  }
+  if (st != PROX_OK) { prox_ffn_destroy(h); return st; }
+  *out = h;
+  return PROX_OK;
+}
+
+void prox_ffn_destroy(prox_ffn_t* h) {
+  if (!h) return;
+  free_packed(h);
+  cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
+  cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
+  cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters);
+  cudaFree(h->x_stage); cudaFree(h->y_stage);
+  if (h->prof) {
+    for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    delete h->prof;
+  }
+  delete h;
+}
+
+prox_status_t prox_quantize_proxy(prox_ffn_t* h, int bits, int group_size, void* stream) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  if (bits != 4 && bits != 8) return PROX_ERR_UNSUPPORTED;
+  if (group_size != 0 && group_size != 128) return PROX_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  const int G = group_size == 0 ? D : group_size;
+  prox_status_t s = alloc_packed(h, bits, G);
+  if (s != PROX_OK) { free_packed(h); return s; }
+  const int ngroups = D / G;
+  {
+    const long long warps = 2ll * F * ngroups;
+    const long long threads = warps * 32;
+    const int bs = 256;
+    proxy_scale_kernel<<<(unsigned)((threads + bs - 1) / bs), bs, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16*>(h->wg), reinterpret_cast<const __nv_bfloat16*>(h->wu), D,
+        F, G, bits, h->S, h->s_plain);
+    h->launches++;
+    CK(cudaGetLastError());
+  }
+  {
+    const long long total = (long long)(F / ch_per_chunk(bits)) * 4 * D;
+    const int bs = 256;
+    proxy_pack_kernel<<<(unsigned)((total + bs - 1) / bs), bs, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16*>(h->wg), reinterpret_cast<const __nv_bfloat16*>(h->wu), D,
+        F, G, bits, h->s_plain, reinterpret_cast<uint32_t*>(h->P));
+    h->launches++;
+    CK(cudaGetLastError());
+  }
+  {
+    dim3 grid((F + 31) / 32, (D + 31) / 32), block(32, 8);
+    transpose_bf16_kernel<<<grid, block, 0, st>>>(h->wd, h->wdt, D, F);
+    h->launches++;
+    CK(cudaGetLastError());
+  }
+  h->quantized = true;
+  return PROX_OK;
+}
+
+prox_status_t prox_input_topk(prox_ffn_t* h, const void* x, int B, int k1, int32_t* idx, void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!idx || k1 < 1 || k1 > h->cfg.d_model) return PROX_ERR_INVALID_ARG;
+  return launch_input_select(h, x, B, k1, 0.f, 0, idx, k1, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x, int B, int k1, int k2, int32_t* sel,
+                               float* scores, void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!sel) return PROX_ERR_INVALID_ARG;
+  if (k1 < 1 || k1 > h->cfg.d_model || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model;
+  float* sc = scores ? scores : h->scores;
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, sc, st)) != PROX_OK) return s;
+  return launch_channel_select(h, sc, B, k2, 0.f, 0, sel, k2, nullptr, st);
+}
+
+prox_status_t prox_stage2_ffn(prox_ffn_t* h, const void* x, int B, const int32_t* sel, int k2, void* y,
+                              void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!sel || !y || !aligned16(y)) return PROX_ERR_INVALID_ARG;
+  if (k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  return launch_stage2(h, x, B, sel, k2, nullptr, k2, y, static_cast<cudaStream_t>(stream));
+}
+
+prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int k2, void* y, void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!y || !aligned16(y)) return PROX_ERR_INVALID_ARG;
+  if (k1 < 1 || k1 > h->cfg.d_model || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
+  if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
+  return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
+}
+
+prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, int k1, int k2,
+                                    void* y_host, void* stream) {
+  if (!h || !x_host || !y_host) return PROX_ERR_INVALID_ARG;
+  if (B < 1 || B > h->cfg.max_batch) return PROX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t D = h->cfg.d_model;
+  const size_t ybytes = (size_t)B * D * (h->cfg.out_dtype ? 4 : 2);
+  CK(cudaMemcpyAsync(h->x_stage, x_host, (size_t)B * D * 2, cudaMemcpyHostToDevice, st));
+  prox_status_t s = prox_ffn_forward(h, h->x_stage, B, k1, k2, h->y_stage, stream);
+  if (s != PROX_OK) return s;
+  CK(cudaMemcpyAsync(y_host, h->y_stage, ybytes, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return PROX_OK;
+}
+
+// ---- threshold variant ------------------------------------------------------
+namespace {
+__global__ void count_accum_kernel(const int* cnt_x, const int* cnt_s, int B, unsigned long long* c) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    unsigned long long a = 0, s = 0;
+    for (int b = 0; b < B; ++b) { a += (unsigned long long)cnt_x[b]; s += (unsigned long long)cnt_s[b]; }
+    c[0] += (unsigned long long)B; c[1] += a; c[2] += s;
+  }
+}
+}  // namespace
+
+prox_status_t prox_stage1_mask_threshold(prox_ffn_t* h, const void* x, int B, float tau_x, float tau_s,
+                                         int32_t* sel, int32_t* count, float* scores, void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!sel || !count) return PROX_ERR_INVALID_ARG;
+  if (!(tau_x >= 0.f) || !(tau_s >= 0.f)) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  float* sc = scores ? scores : h->scores;
+  if ((s = launch_input_select(h, x, B, 0, tau_x, 1, h->idx_x, D, h->cnt_x, st)) != PROX_OK) return s;
+  if ((s = launch_proxy(h, x, B, h->idx_x, D, h->cnt_x, D, sc, st)) != PROX_OK) return s;
+  if ((s = launch_channel_select(h, sc, B, 0, tau_s, 1, sel, F, count, st)) != PROX_OK) return s;
+  count_accum_kernel<<<1, 32, 0, st>>>(h->cnt_x, count, B, h->counters);
+  h->launches++;
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+prox_status_t prox_stage2_ffn_var(prox_ffn_t* h, const void* x, int B, const int32_t* sel,
+                                  const int32_t* count, void* y, void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!sel || !count || !y || !aligned16(y)) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  return launch_stage2(h, x, B, sel, h->cfg.d_ff, count, h->cfg.d_ff, y, static_cast<cudaStream_t>(stream));
+}
+
+prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x, int B, float tau_x, float tau_s,
+                                         void* y, void* stream) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  prox_status_t s = prox_stage1_mask_threshold(h, x, B, tau_x, tau_s, h->sel, h->cnt_s, nullptr, stream);
+  if (s != PROX_OK) return s;
+  return prox_stage2_ffn_var(h, x, B, h->sel, h->cnt_s, y, stream);
+}
+
+prox_status_t prox_runtime_sparsity(prox_ffn_t* h, double alpha, int64_t* tokens, double* s1_hat,
+                                    double* s2_hat, double* e_hat, int reset) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  unsigned long long c[4] = {0, 0, 0, 0};
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(c, h->counters, sizeof(c), cudaMemcpyDeviceToHost));
+  if (reset) CK(cudaMemset(h->counters, 0, sizeof(c)));
+  const double n = (double)c[0];
+  const double s1 = n > 0 ? 1.0 - (double)c[1] / (n * h->cfg.d_model) : 0.0;
+  const double s2 = n > 0 ? 1.0 - (double)c[2] / (n * h->cfg.d_ff) : 0.0;
+  if (tokens) *tokens = (int64_t)c[0];
+  if (s1_hat) *s1_hat = s1;
+  if (s2_hat) *s2_hat = s2;
+  if (e_hat) *e_hat = s2 - 2.0 * alpha * (1.0 - s1) / 3.0;
+  return PROX_OK;
+}
+
+// ---- host helpers -----------------------------------------------------------
+prox_status_t prox_allocate_budget(double e, double alpha, double s_ref, double s1_min, double s1_max,
+                                   double* s1, double* s2) {
+  if (!s1 || !s2) return PROX_ERR_INVALID_ARG;
+  if (!(alpha > 0.0) || !(s1_min <= s1_max) || !std::isfinite(e) || !std::isfinite(s_ref))
+    return PROX_ERR_INVALID_ARG;
+  double b = s_ref;
+  double a = 1.0 - (b - e) * 3.0 / (2.0 * alpha);
+  if (a < s1_min || a > s1_max) {
+    a = a < s1_min ? s1_min : s1_max;
+    b = e + 2.0 * alpha * (1.0 - a) / 3.0;
+  }
+  *s1 = a;
+  *s2 = b;
+  return PROX_OK;
+}
+
+prox_status_t prox_sparsity_to_k(double s, int dim, int* k) {
+  if (!k || dim < 1 || !std::isfinite(s)) return PROX_ERR_INVALID_ARG;
+  double v = std::floor((1.0 - s) * (double)dim + 0.5);
+  if (v < 1.0) v = 1.0;
+  if (v > (double)dim) v = (double)dim;
+  *k = (int)v;
+  return PROX_OK;
+}
+
+prox_status_t prox_algorithmic_bytes(const prox_ffn_t* h, int rows_in, int rows_ch, int64_t* stage1,
+                                     int64_t* gate_up, int64_t* down, int64_t* activations) {
+  if (!h || rows_in < 0 || rows_ch < 0) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  const int64_t D = h->cfg.d_model, F = h->cfg.d_ff;
+  const int64_t ngroups = D / h->group;
+  if (stage1) *stage1 = (int64_t)rows_in * F * h->bits / 4 + 2 * ngroups * F * 2;
+  if (gate_up) *gate_up = 2 * (int64_t)rows_ch * D * 2;
+  if (down) *down = (int64_t)rows_ch * D * 2;
+  if (activations) *activations = 4 * D + 8 * F + 16 * (int64_t)rows_ch + (h->cfg.out_dtype ? 4 : 2) * D;
+  return PROX_OK;
+}
+
+// ---- export / save / load ---------------------------------------------------
+prox_status_t prox_proxy_export(prox_ffn_t* h, int which, int8_t* q_host, float* scale_host) {
+  if (!h || !q_host || !scale_host || (which != 0 && which != 1)) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  CK(cudaDeviceSynchronize());
+  const int D = h->cfg.d_model, F = h->cfg.d_ff, bits = h->bits;
+  const int CH = ch_per_chunk(bits), nchunks = F / CH, ngroups = D / h->group;
+  std::vector<uint32_t> P;
+  try { P.resize(h->p_bytes / 4); } catch (...) { return PROX_ERR_OOM; }
+  CK(cudaMemcpy(P.data(), h->P, h->p_bytes, cudaMemcpyDeviceToHost));
+  const int per_word = bits == 4 ? 8 : 4;
+  const uint32_t mask = bits == 4 ? 0xFu : 0xFFu;
+  const int off = bits == 4 ? 8 : 128;
+  for (int i = 0; i < D; ++i) {
+    const uint32_t* row = P.data() + (size_t)i * nchunks * 4;
+    for (int c = 0; c < nchunks; ++c)
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t w = row[c * 4 + which * 2 + half];
+        for (int m = 0; m < per_word; ++m) {
+          const int j = c * CH + half * per_word + m;
+          q_host[(size_t)j * D + i] = (int8_t)((int)((w >> (m * bits)) & mask) - off);
+        }
+      }
+  }
+  CK(cudaMemcpy(scale_host, h->s_plain + (size_t)which * F * ngroups, (size_t)F * ngroups * sizeof(float),
+                cudaMemcpyDeviceToHost));
+  return PROX_OK;
+}
+
+namespace {
+struct PackHeader {
+  char magic[8];
+  int32_t version, d_model, d_ff, bits, group;
+  uint64_t p_bytes, s_count, wdt_count;
+};
+const char kMagic[8] = {'P', 'R', 'O', 'X', 'P', 'A', 'C', 'K'};
+}  // namespace
+
+prox_status_t prox_pack_save(prox_ffn_t* h, const char* path) {
+  if (!h || !path) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  CK(cudaDeviceSynchronize());
+  const int D = h->cfg.d_model, F = h->cfg.d_ff, ngroups = D / h->group;
+  PackHeader hd;
+  std::memset(&hd, 0, sizeof(hd));
+  std::memcpy(hd.magic, kMagic, 8);
+  hd.version = 1; hd.d_model = D; hd.d_ff = F; hd.bits = h->bits; hd.group = h->group;
+  hd.p_bytes = h->p_bytes; hd.s_count = h->s_count; hd.wdt_count = (uint64_t)F * D;
+  std::vector<char> buf;
+  const size_t sp_bytes = (size_t)2 * F * ngroups * sizeof(float);
+  const size_t biggest = h->p_bytes > hd.wdt_count * 2 ? h->p_bytes : hd.wdt_count * 2;
+  try { buf.resize(biggest > sp_bytes ? biggest : sp_bytes); } catch (...) { return PROX_ERR_OOM; }
+  FILE* f = std::fopen(path, "wb");
+  if (!f) return PROX_ERR_IO;
+  bool ok = std::fwrite(&hd, sizeof(hd), 1, f) == 1;
+  auto dump = [&](const void* dev, size_t bytes) {
+    if (!ok) return;
+    if (cudaMemcpy(buf.data(), dev, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) { ok = false; return; }
+    ok = std::fwrite(buf.data(), 1, bytes, f) == bytes;
+  };
+  dump(h->P, h->p_bytes);
+  dump(h->S, h->s_count * sizeof(__half));
+  dump(h->s_plain, sp_bytes);
+  dump(h->wdt, hd.wdt_count * 2);
+  ok = (std::fclose(f) == 0) && ok;
+  return ok ? PROX_OK : PROX_ERR_IO;
+}
+
+prox_status_t prox_pack_load(prox_ffn_t* h, const char* path, void* stream) {
+  if (!h || !path) return PROX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FILE* f = std::fopen(path, "rb");
+  if (!f) return PROX_ERR_IO;
+  PackHeader hd;
+  if (std::fread(&hd, sizeof(hd), 1, f) != 1 || std::memcmp(hd.magic, kMagic, 8) != 0 || hd.version != 1) {
+    std::fclose(f);
+    return PROX_ERR_IO;
+  }
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  const bool shape_ok = hd.d_model == D && hd.d_ff == F && (hd.bits == 4 || hd.bits == 8) &&
+                        (hd.group == D || hd.group == 128);
+  if (!shape_ok) { std::fclose(f); return PROX_ERR_INVALID_ARG; }
+  prox_status_t s = alloc_packed(h, hd.bits, hd.group);
+  if (s != PROX_OK) { std::fclose(f); free_packed(h); return s; }
+  const int ngroups = D / hd.group;
+  const size_t sp_bytes = (size_t)2 * F * ngroups * sizeof(float);
+  if (hd.p_bytes != h->p_bytes || hd.s_count != h->s_count || hd.wdt_count != (uint64_t)F * D) {
+    std::fclose(f); free_packed(h);
+    return PROX_ERR_IO;
+  }
+  std::vector<char> buf;
+  const size_t biggest = h->p_bytes > (size_t)F * D * 2 ? h->p_bytes : (size_t)F * D * 2;
+  try { buf.resize(biggest > sp_bytes ? biggest : sp_bytes); } catch (...) { std::fclose(f); free_packed(h); return PROX_ERR_OOM; }
+  bool ok = true;
+  cudaError_t ce = cudaSuccess;
+  auto fill = [&](void* dev, size_t bytes) {
+    if (!ok) return;
+    if (std::fread(buf.data(), 1, bytes, f) != bytes) { ok = false; return; }
+    ce = cudaMemcpyAsync(dev, buf.data(), bytes, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) ok = false;
+  };
+  fill(h->P, h->p_bytes);
+  fill(h->S, h->s_count * sizeof(__half));
+  fill(h->s_plain, sp_bytes);
+  fill(h->wdt, (size_t)F * D * 2);
+  std::fclose(f);
+  if (!ok) { free_packed(h); return ce != cudaSuccess ? map_cuda(ce) : PROX_ERR_IO; }
+  h->quantized = true;
+  return PROX_OK;
+}
+
+prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream) {
+  if (!h || !code) return PROX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CK(cudaMemcpyAsync(code, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CK(cudaMemsetAsync(h->dev_status, 0, sizeof(int), st));
+  CK(cudaStreamSynchronize(st));
+  return PROX_OK;
+}
+
+prox_status_t prox_profile_enable(prox_ffn_t* h, int on) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  h->profiling = on != 0;
+  return PROX_OK;
+}
+
+prox_status_t prox_profile_read(prox_ffn_t* h, int64_t* counts, double* ms) {
+  if (!h || !counts || !ms) return PROX_ERR_INVALID_ARG;
+  for (int k = 0; k < PROX_NUM_KERNEL_KINDS; ++k) { counts[k] = 0; ms[k] = 0.0; }
+  prox_status_t st = PROX_OK;
+  for (auto& r : *h->prof) {
+    float t = 0.f;
+    cudaError_t e = cudaEventSynchronize(r.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.a, r.b);
+    if (e == cudaSuccess && r.kind >= 0 && r.kind < PROX_NUM_KERNEL_KINDS) { counts[r.kind]++; ms[r.kind] += t; }
+    else if (e != cudaSuccess) st = PROX_ERR_CUDA;
+    cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+  }
+  h->prof->clear();
+  return st;
+}
+
+prox_status_t prox_launch_count(const prox_ffn_t* h, int64_t* launches) {
+  if (!h || !launches) return PROX_ERR_INVALID_ARG;
+  *launches = h->launches;
+  return PROX_OK;
+}
+
+const char* prox_status_string(prox_status_t s) {
+  switch (s) {
+    case PROX_OK: return "ok";
+    case PROX_ERR_INVALID_ARG: return "invalid argument";
+    case PROX_ERR_UNSUPPORTED: return "unsupported shape or format";
+    case PROX_ERR_NOT_QUANTIZED: return "proxy not quantized yet";
+    case PROX_ERR_CUDA: return "CUDA runtime error";
+    case PROX_ERR_OOM: return "out of memory";
+    case PROX_ERR_TIMEOUT: return "device-side wait timed out";
+    case PROX_ERR_IO: return "file I/O error";
+  }
+  return "unknown status";
+}
+
+const char* prox_version(void) { return "libprox 0.1 (sm_100a)"; }
+
+}  // extern "C"

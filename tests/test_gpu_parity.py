@@ -1,0 +1,320 @@
+"""GPU parity: libprox (through the C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Tolerances (written here, derived in
+the design doc): integer work (quantizer codes, input mask) bit-exact; channel masks
+identical outside a 1e-3 relative band around the k2-th oracle score; outputs
+within 2e-2 * RMS(y_oracle)."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import prox_oracle as po
+from paper_2607_27591_b200 import inputs
+from tests.gpu_common import Problem, check_mask, check_y
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pb():
+    entry.build()
+    from paper_2607_27591_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def toy(pb):
+    wl, wg, wu, wd, x = inputs.make_workload("toy")
+    p = Problem(pb, wg, wu, wd, x, max_batch=8)
+    yield wl, p
+    p.close()
+
+
+# ---------------------------------------------------------------- quantizer
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0), (8, 128)])
+def test_quantizer_bit_exact(pb, toy, bits, group):
+    wl, p = toy
+    _, _, (qg, sg, qu, su) = p.quantize(bits, group)
+    ng = 1 if group == 0 else p.D // group
+    for which, (q_ref, s_ref) in enumerate(((qg, sg), (qu, su))):
+        q = np.empty((p.F, p.D), dtype=np.int8)
+        s = np.empty((p.F, ng), dtype=np.float32)
+        pb.prox_proxy_export(p.h, which, q, s)
+        assert np.array_equal(s, s_ref.astype(np.float32)), "scales differ"
+        assert np.array_equal(q, q_ref), f"{(q != q_ref).sum()} codes differ"
+
+
+def test_quantizer_zero_rows_and_ragged_shape(pb):
+    wg, wu, wd, x = inputs.make_small(384, 320, 2, seed=5)      # F = 320: last strip is ragged
+    wg[7, :] = 0
+    wu[9, 128:256] = 0
+    p = Problem(pb, wg, wu, wd, x)
+    try:
+        for bits, group in ((4, 0), (4, 128), (8, 128)):
+            _, _, (qg, sg, qu, su) = p.quantize(bits, group)
+            ng = 1 if group == 0 else p.D // group
+            for which, (q_ref, s_ref) in enumerate(((qg, sg), (qu, su))):
+                q = np.empty((p.F, p.D), dtype=np.int8)
+                s = np.empty((p.F, ng), dtype=np.float32)
+                pb.prox_proxy_export(p.h, which, q, s)
+                assert np.array_equal(s, s_ref.astype(np.float32)) and np.array_equal(q, q_ref)
+    finally:
+        p.close()
+
+
+# --------------------------------------------------------------- input mask
+def test_input_topk_exact(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    for k1 in (1, 2, 31, 461, p.D - 1, p.D):
+        idx = torch.empty(8, k1, dtype=torch.int32, device="cuda")
+        pb.prox_input_topk(p.h, p.t_x[:8], 8, k1, idx)
+        got = idx.cpu().numpy()
+        for t in range(8):
+            assert np.array_equal(got[t], po.input_topk(p.x[t], k1)), (k1, t)
+
+
+def test_input_topk_ties(pb, toy):
+    """bf16 magnitudes tie often; lower index must win."""
+    wl, p = toy
+    vals = np.array([1.0, -1.0, 0.5, 2.0, -2.0, 0.0, -0.0, 1.0], dtype=np.float32)
+    x = np.tile(vals, p.D // 8)[None, :]
+    bits = inputs.f32_to_bf16_bits(x)
+    from tests.gpu_common import dev_bf16
+    tx = dev_bf16(bits)
+    for k1 in (1, 64, 65, 128, 129, 300, p.D - 3):
+        idx = torch.empty(1, k1, dtype=torch.int32, device="cuda")
+        pb.prox_input_topk(p.h, tx, 1, k1, idx)
+        assert np.array_equal(idx.cpu().numpy()[0], po.input_topk(x[0].astype(np.float64), k1)), k1
+
+
+# ------------------------------------------------------------------ Stage 1
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0)])
+def test_stage1_mask_toy(pb, toy, bits, group):
+    wl, p = toy
+    p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    sel = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+    sc = torch.empty(1, p.F, dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for t in range(p.x.shape[0]):
+        pb.prox_stage1_mask(p.h, p.t_x[t], 1, k1, k2, sel, sc)
+        torch.cuda.synchronize()
+        idx, score, sel_ref, thr = p.oracle_stage1(t, k1, k2)
+        check_mask(sel.cpu().numpy()[0].astype(np.int64), score, sel_ref, thr, k2, p.F)
+        got = sc.cpu().numpy()[0].astype(np.float64)
+        worst = max(worst, float(np.max(np.abs(got - score)) / thr))
+    assert worst < 2e-4, worst          # fp32 accumulation + fast exp, relative to the threshold score
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("k1,k2", [(512, 1536), (1, 1), (512, 1), (17, 1535), (300, 768)])
+def test_stage1_edge_budgets(pb, toy, k1, k2):
+    wl, p = toy
+    p.quantize(4, 0)
+    sel = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+    for t in (0, 5):
+        pb.prox_stage1_mask(p.h, p.t_x[t], 1, k1, k2, sel, None)
+        idx, score, sel_ref, thr = p.oracle_stage1(t, k1, k2)
+        check_mask(sel.cpu().numpy()[0].astype(np.int64), score, sel_ref, thr, k2, p.F)
+
+
+# ------------------------------------------------------------------ Stage 2
+def test_stage2_given_mask(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    rng = np.random.default_rng(0)
+    for k2 in (1, 7, 461, 1000, p.F):
+        for t in (0, 3):
+            sel = np.sort(rng.choice(p.F, size=k2, replace=False)).astype(np.int32)
+            y = p.y_empty()
+            pb.prox_stage2_ffn(p.h, p.t_x[t], 1, torch.from_numpy(sel).cuda(), k2, y)
+            torch.cuda.synchronize()
+            y_ref, _ = po.stage2(p.x[t], sel, p.wg, p.wu, p.wd)
+            rel = check_y(y.cpu().numpy()[0], y_ref)
+            assert rel < 1e-4, rel        # fp32 accumulate, fp32 output: far inside the bound
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+def test_stage2_dense_special_case(pb, toy):
+    """k2 = d_ff: the path is the dense SwiGLU FFN (Sec. 2.1)."""
+    wl, p = toy
+    p.quantize(4, 0)
+    y = p.y_empty()
+    pb.prox_ffn_forward(p.h, p.t_x[1], 1, 100, p.F, y)
+    y_ref, _ = po.dense_ffn(p.x[1], p.wg, p.wu, p.wd)
+    assert check_y(y.cpu().numpy()[0], y_ref) < 1e-4
+
+
+def test_stage2_bf16_output(pb):
+    wl, wg, wu, wd, x = inputs.make_workload("toy", n_tokens=2)
+    p = Problem(pb, wg, wu, wd, x, out_dtype=0)
+    try:
+        p.quantize(4, 0)
+        sel = np.arange(0, p.F, 3, dtype=np.int32)
+        y = p.y_empty()
+        pb.prox_stage2_ffn(p.h, p.t_x[0], 1, torch.from_numpy(sel).cuda(), len(sel), y)
+        y_ref, _ = po.stage2(p.x[0], sel, p.wg, p.wu, p.wd)
+        got = y.float().cpu().numpy()[0]
+        check_y(got, y_ref)
+        # single rounding: equals bf16(oracle) up to one bf16 ulp where fp32 rounding straddles a tie
+        want = inputs.bf16_bits_to_f32(po.f64_to_bf16_bits(y_ref))
+        assert np.mean(got == want) > 0.99
+        assert np.max(np.abs(got - want) / np.maximum(np.abs(want), 1e-30)) <= 2.0 ** -7
+    finally:
+        p.close()
+
+
+def test_stage2_out_of_range_channel_is_skipped_and_recorded(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    sel = np.array([3, 10, p.F + 5, 2 ** 30], dtype=np.int32)
+    y = p.y_empty()
+    pb.prox_stage2_ffn(p.h, p.t_x[0], 1, torch.from_numpy(sel).cuda(), 4, y)
+    assert pb.prox_last_device_status(p.h) & 1
+    assert pb.prox_last_device_status(p.h) == 0      # reading clears
+    y_ref, _ = po.stage2(p.x[0], sel[:2], p.wg, p.wu, p.wd)
+    check_y(y.cpu().numpy()[0], y_ref)
+
+
+# --------------------------------------------------------------- whole path
+def _forward_check(pb, p, t, k1, k2, B=1):
+    y = p.y_empty(B)
+    sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+    xb = p.t_x[t:t + B]
+    pb.prox_stage1_mask(p.h, xb, B, k1, k2, sel)
+    pb.prox_ffn_forward(p.h, xb, B, k1, k2, y)
+    torch.cuda.synchronize()
+    sel_np, y_np = sel.cpu().numpy().astype(np.int64), y.float().cpu().numpy()
+    nd = 0
+    for b in range(B):
+        idx, score, sel_ref, thr = p.oracle_stage1(t + b, k1, k2)
+        nd += check_mask(sel_np[b], score, sel_ref, thr, k2, p.F)
+        y_ref, _ = po.stage2(p.x[t + b], sel_np[b], p.wg, p.wu, p.wd)
+        check_y(y_np[b], y_ref)
+    return nd
+
+
+def test_forward_toy_all_tokens(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    k1, k2 = wl.points[50]
+    for t in range(p.x.shape[0]):
+        _forward_check(pb, p, t, k1, k2)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("B", [2, 4, 8])
+def test_forward_batched_per_token_masks(pb, toy, B):
+    wl, p = toy
+    p.quantize(4, 128)
+    k1, k2 = wl.points[50]
+    _forward_check(pb, p, 3, k1, k2, B=B)
+
+
+def test_forward_host_buffers(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    k1, k2 = wl.points[50]
+    xh = torch.from_numpy(p.bits["x"][2:3].view(np.int16)).view(torch.bfloat16).pin_memory()
+    yh = torch.empty(1, p.D, dtype=torch.float32).pin_memory()
+    pb.prox_ffn_forward_host(p.h, xh, 1, k1, k2, yh)
+    y = p.y_empty()
+    pb.prox_ffn_forward(p.h, p.t_x[2], 1, k1, k2, y)
+    torch.cuda.synchronize()
+    # same kernels, same mask; the fp32 atomics of the down projection may add in another order
+    assert torch.allclose(yh, y.cpu(), rtol=0, atol=1e-5 * float(y.abs().max()))
+
+
+def test_calls_are_repeatable(pb, toy):
+    """Scratch (tickets, accumulators) is left clean: the same call twice gives the same bits
+    for the mask, and outputs that differ only by fp32 atomic ordering."""
+    wl, p = toy
+    p.quantize(4, 0)
+    k1, k2 = wl.points[50]
+    s1 = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+    s2 = torch.empty_like(s1)
+    y1, y2 = p.y_empty(), p.y_empty()
+    pb.prox_stage1_mask(p.h, p.t_x[4], 1, k1, k2, s1)
+    pb.prox_ffn_forward(p.h, p.t_x[4], 1, k1, k2, y1)
+    pb.prox_stage1_mask(p.h, p.t_x[4], 1, k1, k2, s2)
+    pb.prox_ffn_forward(p.h, p.t_x[4], 1, k1, k2, y2)
+    assert torch.equal(s1, s2)
+    assert torch.allclose(y1, y2, rtol=0, atol=1e-5 * float(y1.abs().max()))
+
+
+# --------------------------------------------------------- threshold variant
+def test_threshold_variant(pb, toy):
+    wl, p = toy
+    dg, du, _ = p.quantize(4, 0)
+    k1, k2 = wl.points[50]
+    t = 6
+    idx, score, sel_ref, thr = p.oracle_stage1(t, k1, k2)
+    mags = np.sort(np.abs(p.x[t]))[::-1]
+    tau_x = float((mags[k1 - 1] + mags[k1]) / 2) if mags[k1 - 1] != mags[k1] else float(mags[k1 - 1])
+    idx_t = po.input_threshold(p.x[t], np.float32(tau_x))
+    score_t = po.proxy_scores(p.x[t], idx_t, dg, du)
+    srt = np.sort(score_t)[::-1]
+    tau_s = float(np.float32((srt[k2 - 1] + srt[k2]) / 2))
+    sel_t = po.channel_threshold(score_t, tau_s)
+    sel = torch.empty(1, p.F, dtype=torch.int32, device="cuda")
+    cnt = torch.empty(1, dtype=torch.int32, device="cuda")
+    y = p.y_empty()
+    pb.prox_runtime_sparsity(p.h, reset=True)
+    pb.prox_stage1_mask_threshold(p.h, p.t_x[t], 1, tau_x, tau_s, sel, cnt)
+    pb.prox_stage2_ffn_var(p.h, p.t_x[t], 1, sel, cnt, y)
+    torch.cuda.synchronize()
+    n = int(cnt.item())
+    got = sel.cpu().numpy()[0, :n].astype(np.int64)
+    near = np.abs(score_t - tau_s) <= 1e-3 * tau_s
+    assert np.all(near[np.setxor1d(got, sel_t)])
+    y_ref, _ = po.stage2(p.x[t], got, p.wg, p.wu, p.wd)
+    check_y(y.cpu().numpy()[0], y_ref)
+    tok, s1h, s2h, eh = pb.prox_runtime_sparsity(p.h)
+    assert tok == 1 and abs(s1h - (1 - len(idx_t) / p.D)) < 1e-12 and abs(s2h - (1 - n / p.F)) < 1e-12
+    assert abs(eh - po.effective_sparsity(s1h, s2h)) < 1e-12
+    y2 = p.y_empty()
+    pb.prox_ffn_forward_threshold(p.h, p.t_x[t], 1, tau_x, tau_s, y2)
+    assert torch.allclose(y, y2, rtol=0, atol=1e-5 * float(y.abs().max()))
+
+
+# ------------------------------------------------------------- pack save/load
+def test_pack_save_load_roundtrip(pb, toy, tmp_path):
+    wl, p = toy
+    p.quantize(4, 128)
+    k1, k2 = wl.points[50]
+    path = str(tmp_path / "layer0.proxpack")
+    pb.prox_pack_save(p.h, path)
+    sel_a = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+    pb.prox_stage1_mask(p.h, p.t_x[0], 1, k1, k2, sel_a)
+    p2 = Problem(pb, p.bits["wg"], p.bits["wu"], p.bits["wd"], p.bits["x"])
+    try:
+        with pytest.raises(pb.ProxError):
+            pb.prox_stage1_mask(p2.h, p2.t_x[0], 1, k1, k2, sel_a)      # not quantized yet
+        pb.prox_pack_load(p2.h, path)
+        sel_b = torch.empty_like(sel_a)
+        pb.prox_stage1_mask(p2.h, p2.t_x[0], 1, k1, k2, sel_b)
+        assert torch.equal(sel_a, sel_b)
+        with pytest.raises(pb.ProxError):
+            pb.prox_pack_load(p2.h, str(tmp_path / "missing"))
+    finally:
+        p2.close()
+
+
+def test_device_argument_validation(pb, toy):
+    wl, p = toy
+    p.quantize(4, 0)
+    y = p.y_empty()
+    sel = torch.empty(1, 8, dtype=torch.int32, device="cuda")
+    R = pb.raw
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 0, 1, 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 9, 1, 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 1, 0, 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 1, p.D + 1, 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 1, 1, p.F + 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr() + 2, 1, 1, 1, y.data_ptr(), None) == 1
+    assert R("prox_ffn_forward")(p.h, p.t_x.data_ptr(), 1, 1, 1, None, None) == 1
+    assert R("prox_stage1_mask")(p.h, p.t_x.data_ptr(), 1, 1, 1, None, None, None) == 1
+    assert R("prox_stage2_ffn")(p.h, p.t_x.data_ptr(), 1, sel.data_ptr(), 0, y.data_ptr(), None) == 1
+    assert R("prox_quantize_proxy")(p.h, 3, 0, None) == 2
+    assert R("prox_quantize_proxy")(p.h, 4, 64, None) == 2

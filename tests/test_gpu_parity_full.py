@@ -1,0 +1,88 @@
+"""GPU parity at the benchmark shapes (full d_model / d_ff of every workload,
+the launch configuration bench.py times), on a few tokens each so that the
+oracle finishes in seconds."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import prox_oracle as po
+from paper_2607_27591_b200 import inputs
+from tests.gpu_common import Problem, check_mask, check_y
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pb():
+    entry.build()
+    from paper_2607_27591_b200 import binding
+    return binding
+
+
+def _run(pb, name, n_tok, cases, batches=(1,)):
+    wl, wg, wu, wd, x = inputs.make_workload(name, n_tokens=n_tok)
+    p = Problem(pb, wg, wu, wd, x, max_batch=max(batches))
+    try:
+        for (bits, group), e in cases:
+            p.quantize(bits, group)
+            k1, k2 = wl.points[e]
+            for B in batches:
+                for t0 in range(0, n_tok - B + 1, B):
+                    y = p.y_empty(B)
+                    sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+                    xb = p.t_x[t0:t0 + B]
+                    pb.prox_stage1_mask(p.h, xb, B, k1, k2, sel)
+                    pb.prox_ffn_forward(p.h, xb, B, k1, k2, y)
+                    torch.cuda.synchronize()
+                    sel_np, y_np = sel.cpu().numpy().astype(np.int64), y.cpu().numpy()
+                    for b in range(B):
+                        idx, score, sel_ref, thr = p.oracle_stage1(t0 + b, k1, k2)
+                        check_mask(sel_np[b], score, sel_ref, thr, k2, p.F)
+                        y_ref, _ = po.stage2(p.x[t0 + b], sel_np[b], p.wg, p.wu, p.wd)
+                        check_y(y_np[b], y_ref)
+                    if B == 1:
+                        # Stage 2 alone, fed the oracle's own mask
+                        ys = p.y_empty(1)
+                        pb.prox_stage2_ffn(p.h, p.t_x[t0], 1, torch.from_numpy(sel_ref.astype(np.int32)).cuda(), k2, ys)
+                        y_ref, _ = po.stage2(p.x[t0], sel_ref, p.wg, p.wu, p.wd)
+                        check_y(ys.cpu().numpy()[0], y_ref)
+            assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
+
+
+def test_qwen3_0p6b_all_sparsities(pb):
+    _run(pb, "qwen3_0p6b", 6, [((4, 0), 50), ((4, 0), 70), ((4, 0), 90)])
+
+
+def test_qwen3_8b(pb):
+    _run(pb, "qwen3_8b", 4, [((4, 128), 70)])
+
+
+def test_llama3_8b_formats_and_batches(pb):
+    _run(pb, "llama3_8b", 8, [((8, 0), 70), ((4, 128), 70), ((4, 128), 40)], batches=(1, 4, 8))
+
+
+def test_llama3_70b(pb):
+    _run(pb, "llama3_70b", 8, [((4, 0), 70), ((4, 128), 70)], batches=(1, 8))
+
+
+def test_llama3_70b_s1_sweep(pb):
+    wl, wg, wu, wd, x = inputs.make_workload("llama3_70b", n_tokens=1)
+    p = Problem(pb, wg, wu, wd, x)
+    try:
+        p.quantize(4, 0)
+        for k1, k2 in wl.extra["s1_sweep"][::3]:
+            y = p.y_empty()
+            sel = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+            pb.prox_stage1_mask(p.h, p.t_x[0], 1, k1, k2, sel)
+            pb.prox_ffn_forward(p.h, p.t_x[0], 1, k1, k2, y)
+            torch.cuda.synchronize()
+            sel_np = sel.cpu().numpy()[0].astype(np.int64)
+            idx, score, sel_ref, thr = p.oracle_stage1(0, k1, k2)
+            check_mask(sel_np, score, sel_ref, thr, k2, p.F)
+            y_ref, _ = po.stage2(p.x[0], sel_np, p.wg, p.wu, p.wd)
+            check_y(y.cpu().numpy()[0], y_ref)
+    finally:
+        p.close()
