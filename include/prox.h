@@ -118,6 +118,23 @@ prox_status_t prox_stage2_ffn(prox_ffn_t* h, const void* x_dev, int B, const int
 prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x_dev, int B, int k1, int k2,
                                void* y_dev, void* stream);
 
+/* For B = 1 prox_ffn_forward runs the whole path as ONE persistent kernel
+ * (cooperative launch, one block per SM, one grid-wide barrier with a bounded
+ * wait between Stage 1 and Stage 2); prox_ffn_set_fused(h, 0) selects the
+ * kernel-per-step path instead (always used for B > 1).  If a bounded wait
+ * ever expires the kernel leaves, y is not written and
+ * prox_last_device_status reports bit 4. */
+prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
+
+/* Launch plan of the persistent kernel for budgets (k1, k2), for diagnostics:
+ * info[8] (host) = {usable, grid blocks, row split, dynamic shared bytes, ring
+ * slots, registers per thread, static shared bytes, co-resident blocks per SM}. */
+prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* info_host);
+
+/* Copy the channel mask of the most recent prox_ffn_forward call (top-k rule)
+ * into sel_dev, dev int32 [B, k2], ascending per token.  Enqueued on stream. */
+prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev, void* stream);
+
 /* Same as prox_ffn_forward with HOST buffers: copies x (host bf16 [B, D]) to
  * the device, runs the path, copies y back and synchronises the stream before
  * returning.  Pinned host memory makes the copies asynchronous w.r.t. other
@@ -198,6 +215,9 @@ prox_status_t prox_launch_count(const prox_ffn_t* h, int64_t* launches);
 
 void prox_ffn_destroy(prox_ffn_t* h);
 const char* prox_status_string(prox_status_t s);
+/* Text of the CUDA error behind the calling thread's most recent PROX_ERR_CUDA /
+ * PROX_ERR_OOM ("" if none). */
+const char* prox_last_cuda_error(void);
 const char* prox_version(void);
 
 #ifdef __cplusplus

@@ -24,7 +24,9 @@ STATUS_NAMES = {
 class ProxError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({prox_status_string(status)})")
+        detail = _lib.prox_last_cuda_error().decode() if status in (4, 5) else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({prox_status_string(status)})"
+                         + (f": {detail}" if detail else ""))
 
 
 class ProxFFNConfig(C.Structure):
@@ -60,6 +62,9 @@ _SIGS = {
                                C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
     "prox_last_device_status": [_vp, C.POINTER(C.c_int32), _vp],
     "prox_launch_count": [_vp, C.POINTER(C.c_int64)],
+    "prox_ffn_set_fused": [_vp, _i],
+    "prox_fused_kernel_info": [_vp, _i, _i, C.POINTER(C.c_int32)],
+    "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
     "prox_profile_enable": [_vp, _i],
     "prox_profile_read": [_vp, C.POINTER(C.c_int64), C.POINTER(_d)],
 }
@@ -71,10 +76,12 @@ _lib.prox_ffn_destroy.argtypes = [_vp]
 _lib.prox_ffn_destroy.restype = None
 _lib.prox_status_string.argtypes = [C.c_int]
 _lib.prox_status_string.restype = C.c_char_p
+_lib.prox_last_cuda_error.argtypes = []
+_lib.prox_last_cuda_error.restype = C.c_char_p
 _lib.prox_version.argtypes = []
 _lib.prox_version.restype = C.c_char_p
 
-EXPORTED = tuple(_SIGS) + ("prox_ffn_destroy", "prox_status_string", "prox_version")
+EXPORTED = tuple(_SIGS) + ("prox_ffn_destroy", "prox_status_string", "prox_version", "prox_last_cuda_error")
 
 
 def _ptr(obj) -> Optional[int]:
@@ -131,6 +138,21 @@ def prox_stage2_ffn(handle: int, x, B: int, sel, k2: int, y, stream=None) -> Non
 
 def prox_ffn_forward(handle: int, x, B: int, k1: int, k2: int, y, stream=None) -> None:
     _check(_lib.prox_ffn_forward(handle, _ptr(x), B, k1, k2, _ptr(y), _ptr(stream)), "prox_ffn_forward")
+
+
+def prox_ffn_set_fused(handle: int, on: int) -> None:
+    _check(_lib.prox_ffn_set_fused(handle, int(on)), "prox_ffn_set_fused")
+
+
+def prox_fused_kernel_info(handle: int, k1: int, k2: int) -> dict:
+    info = (C.c_int32 * 8)()
+    _check(_lib.prox_fused_kernel_info(handle, k1, k2, info), "prox_fused_kernel_info")
+    keys = ("usable", "grid", "ksplit", "smem_bytes", "ring_slots", "registers", "static_smem", "blocks_per_sm")
+    return dict(zip(keys, list(info)))
+
+
+def prox_ffn_last_mask(handle: int, B: int, k2: int, sel, stream=None) -> None:
+    _check(_lib.prox_ffn_last_mask(handle, B, k2, _ptr(sel), _ptr(stream)), "prox_ffn_last_mask")
 
 
 def prox_ffn_forward_host(handle: int, x_host, B: int, k1: int, k2: int, y_host, stream=None) -> None:

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "prox_kernels.cuh"
+#include "prox_fused.cuh"
 
 using namespace prox;
 
@@ -45,6 +46,11 @@ struct prox_ffn {
   float* yacc;              // [maxB][D]
   int* dev_status;
   unsigned long long* counters;  // [0] tokens, [1] kept inputs, [2] kept channels
+  unsigned* syncbuf;        // fused kernel: [0..2047] score histogram, [2048] barrier count,
+                            // [2049] barrier generation, [2050] finish ticket
+  int smem_optin;           // largest dynamic shared memory a block may ask for
+  int coop;                 // device supports cooperative launch
+  int use_fused;            // batch-1 forward runs as one persistent kernel
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -60,7 +66,11 @@ namespace {
     if (e_ != cudaSuccess) return map_cuda(e_);    \
   } while (0)
 
+thread_local cudaError_t g_last_cuda = cudaSuccess;
+
 prox_status_t map_cuda(cudaError_t e) {
+  g_last_cuda = e;
+  (void)cudaGetLastError();                       // do not leave a sticky-looking launch error behind
   if (e == cudaErrorMemoryAllocation) return PROX_ERR_OOM;
   return PROX_ERR_CUDA;
 }
@@ -214,6 +224,102 @@ prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, i
   return PROX_OK;
 }
 
+// ---- fused persistent kernel (batch 1) ----------------------------------------
+struct FusedPlan {
+  bool ok;
+  int grid, ksplit, nstrips, big_bytes, nslots, xch;
+  size_t smem;
+};
+
+FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
+  FusedPlan pl;
+  std::memset(&pl, 0, sizeof(pl));
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  if (!h->use_fused || !h->coop) return pl;
+  const int G = h->sm_count;
+  const size_t fixed = ((sizeof(FusedSmem) + 127) & ~size_t(127)) + (size_t)4 * D;
+  if ((size_t)h->smem_optin < fixed + (size_t)6 * D + 16384) return pl;
+  pl.big_bytes = (int)(((size_t)h->smem_optin - fixed) & ~size_t(127));
+  pl.nslots = pl.big_bytes / (2 * D);
+  if (pl.nslots > kMaxSlots) pl.nslots = kMaxSlots;
+  if (pl.nslots < 3) return pl;
+  if (pl.big_bytes < kFusedConsumerWarps * 2 * 512) return pl;          // one row per warp buffer
+  if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;  // reduction scratch
+  if ((k2 + G - 1) / G > kMySelCap) return pl;
+  pl.nstrips = nstrips_for(F, h->bits);
+  // row split: fill the grid evenly (items = strips * ksplit run in rounds of G blocks)
+  int best = 1;
+  double best_eff = -1.0;
+  const int ks_cap = k1 / 16 > 1 ? (k1 / 16 < 16 ? k1 / 16 : 16) : 1;
+  for (int ks = 1; ks <= ks_cap; ++ks) {
+    const int items = pl.nstrips * ks;
+    if ((size_t)items * 1024 > h->part_floats) break;
+    const int rounds = (items + G - 1) / G;
+    const double eff = (double)items / ((double)rounds * G);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
+  }
+  pl.ksplit = best;
+  pl.grid = G;
+  pl.xch = (D / 8 + kFusedConsumers - 1) / kFusedConsumers;
+  pl.xch = pl.xch <= 1 ? 1 : (pl.xch == 2 ? 2 : 4);
+  pl.smem = fixed + (size_t)pl.big_bytes;
+  pl.ok = true;
+  return pl;
+}
+
+template <int BITS, int XCH>
+cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
+  static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
+  auto kern = prox_fused_kernel<BITS, XCH>;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(pl.grid);
+  cfg.blockDim = dim3(kFusedThreads);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;
+  at[0].val.cooperative = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, prm);
+}
+
+prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int k1, int k2, void* y,
+                           int* sel_out, cudaStream_t st) {
+  FusedParams prm;
+  std::memset(&prm, 0, sizeof(prm));
+  prm.P = h->P; prm.S = h->S; prm.wg = h->wg; prm.wu = h->wu; prm.wdt = h->wdt;
+  prm.x = static_cast<const uint16_t*>(x); prm.y = y;
+  prm.D = h->cfg.d_model; prm.F = h->cfg.d_ff; prm.k1 = k1; prm.k2 = k2;
+  prm.gshift = (h->group == h->cfg.d_model) ? 31 : 7;
+  prm.out_fp32 = h->cfg.out_dtype;
+  prm.nstrips = pl.nstrips; prm.ksplit = pl.ksplit;
+  prm.part = h->part; prm.ticket = h->ticket; prm.scores = h->scores; prm.ghist = h->syncbuf;
+  prm.sel_out = sel_out; prm.yacc = h->yacc;
+  prm.bar_count = h->syncbuf + 2048; prm.bar_gen = h->syncbuf + 2049; prm.done_ticket = h->syncbuf + 2050;
+  prm.status = h->dev_status;
+  prm.big_bytes = pl.big_bytes; prm.nslots = pl.nslots;
+  cudaError_t e;
+  {
+    LaunchScope ls(h, kKFused, st);
+    if (h->bits == 4) {
+      e = pl.xch == 1 ? launch_fused_t<4, 1>(pl, prm, st)
+        : pl.xch == 2 ? launch_fused_t<4, 2>(pl, prm, st) : launch_fused_t<4, 4>(pl, prm, st);
+    } else {
+      e = pl.xch == 1 ? launch_fused_t<8, 1>(pl, prm, st)
+        : pl.xch == 2 ? launch_fused_t<8, 2>(pl, prm, st) : launch_fused_t<8, 4>(pl, prm, st);
+    }
+  }
+  CK(e);
+  return PROX_OK;
+}
+
 }  // namespace
 
 // ============================================================================
@@ -261,6 +367,11 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   A(dev_alloc(&h->yacc, (size_t)MB * D));
   A(dev_alloc(&h->dev_status, (size_t)1));
   A(dev_alloc(&h->counters, (size_t)4));
+  A(dev_alloc(&h->syncbuf, (size_t)2048 + 64));
+  A(cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
+  A(cudaDeviceGetAttribute(&h->coop, cudaDevAttrCooperativeLaunch, h->device));
+  h->use_fused = 1;
+  if (st == PROX_OK) A(cudaMemset(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned)));
   A(dev_alloc(reinterpret_cast<uint16_t**>(&h->x_stage), (size_t)MB * D));
   A(dev_alloc(reinterpret_cast<float**>(&h->y_stage), (size_t)MB * D));
   if (st == PROX_OK) {
@@ -279,7 +390,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   free_packed(h);
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
-  cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters);
+  cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -367,10 +478,48 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
   if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  if (B == 1) {
+    const FusedPlan pl = plan_fused(h, k1, k2);
+    if (pl.ok) return launch_fused(h, pl, x, k1, k2, y, h->sel, st);
+  }
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
   if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
   return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
+}
+
+prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* info) {
+  if (!h || !info) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  for (int i = 0; i < 8; ++i) info[i] = 0;
+  const FusedPlan pl = plan_fused(h, k1, k2);
+  info[0] = pl.ok ? 1 : 0;
+  if (!pl.ok) return PROX_OK;
+  const void* fn = h->bits == 4
+      ? (pl.xch == 1 ? (const void*)prox_fused_kernel<4, 1> : pl.xch == 2 ? (const void*)prox_fused_kernel<4, 2> : (const void*)prox_fused_kernel<4, 4>)
+      : (pl.xch == 1 ? (const void*)prox_fused_kernel<8, 1> : pl.xch == 2 ? (const void*)prox_fused_kernel<8, 2> : (const void*)prox_fused_kernel<8, 4>);
+  cudaFuncAttributes fa;
+  CK(cudaFuncGetAttributes(&fa, fn));
+  CK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  int nb = 0;
+  CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kFusedThreads, pl.smem));
+  info[1] = pl.grid; info[2] = pl.ksplit; info[3] = (int)pl.smem; info[4] = pl.nslots;
+  info[5] = fa.numRegs; info[6] = (int)fa.sharedSizeBytes; info[7] = nb;
+  return PROX_OK;
+}
+
+prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  h->use_fused = on != 0;
+  return PROX_OK;
+}
+
+prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev, void* stream) {
+  if (!h || !sel_dev || B < 1 || B > h->cfg.max_batch || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  CK(cudaMemcpy2DAsync(sel_dev, (size_t)k2 * sizeof(int), h->sel, (size_t)h->cfg.d_ff * sizeof(int),
+                       (size_t)k2 * sizeof(int), (size_t)B, cudaMemcpyDeviceToDevice,
+                       static_cast<cudaStream_t>(stream)));
+  return PROX_OK;
 }
 
 prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, int k1, int k2,
@@ -609,6 +758,15 @@ prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream
   CK(cudaMemcpyAsync(code, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st));
   CK(cudaMemsetAsync(h->dev_status, 0, sizeof(int), st));
   CK(cudaStreamSynchronize(st));
+  if (*code & kWaitExpired) {
+    // A block gave up on a wait: counters shared between blocks may be left
+    // half-way.  Put every one of them back to its idle state.
+    const int ns_max = nstrips_for(h->cfg.d_ff, 8);
+    CK(cudaMemsetAsync(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned), st));
+    CK(cudaMemsetAsync(h->ticket, 0, (size_t)h->cfg.max_batch * ns_max * sizeof(unsigned), st));
+    CK(cudaMemsetAsync(h->yacc, 0, (size_t)h->cfg.max_batch * h->cfg.d_model * sizeof(float), st));
+    CK(cudaStreamSynchronize(st));
+  }
   return PROX_OK;
 }
 
@@ -652,6 +810,10 @@ const char* prox_status_string(prox_status_t s) {
     case PROX_ERR_IO: return "file I/O error";
   }
   return "unknown status";
+}
+
+const char* prox_last_cuda_error(void) {
+  return g_last_cuda == cudaSuccess ? "" : cudaGetErrorString(g_last_cuda);
 }
 
 const char* prox_version(void) { return "libprox 0.1 (sm_100a)"; }

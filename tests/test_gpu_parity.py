@@ -184,13 +184,17 @@ def _forward_check(pb, p, t, k1, k2, B=1):
     xb = p.t_x[t:t + B]
     pb.prox_stage1_mask(p.h, xb, B, k1, k2, sel)
     pb.prox_ffn_forward(p.h, xb, B, k1, k2, y)
+    used = torch.empty_like(sel)                     # the mask the forward call itself built
+    pb.prox_ffn_last_mask(p.h, B, k2, used)
     torch.cuda.synchronize()
-    sel_np, y_np = sel.cpu().numpy().astype(np.int64), y.float().cpu().numpy()
+    sel_np, used_np, y_np = (sel.cpu().numpy().astype(np.int64), used.cpu().numpy().astype(np.int64),
+                             y.float().cpu().numpy())
     nd = 0
     for b in range(B):
         idx, score, sel_ref, thr = p.oracle_stage1(t + b, k1, k2)
         nd += check_mask(sel_np[b], score, sel_ref, thr, k2, p.F)
-        y_ref, _ = po.stage2(p.x[t + b], sel_np[b], p.wg, p.wu, p.wd)
+        nd += check_mask(used_np[b], score, sel_ref, thr, k2, p.F)
+        y_ref, _ = po.stage2(p.x[t + b], used_np[b], p.wg, p.wu, p.wd)
         check_y(y_np[b], y_ref)
     return nd
 
@@ -241,6 +245,56 @@ def test_calls_are_repeatable(pb, toy):
     pb.prox_ffn_forward(p.h, p.t_x[4], 1, k1, k2, y2)
     assert torch.equal(s1, s2)
     assert torch.allclose(y1, y2, rtol=0, atol=1e-5 * float(y1.abs().max()))
+
+
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0), (8, 128)])
+def test_fused_and_stepwise_paths_agree(pb, toy, bits, group):
+    """B = 1 runs as one persistent kernel by default; the kernel-per-step path
+    must give the same mask (up to the band) and the same y (up to fp32 order)."""
+    wl, p = toy
+    p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    for t in (0, 9, 31):
+        outs = []
+        for fused in (1, 0):
+            pb.prox_ffn_set_fused(p.h, fused)
+            y = p.y_empty()
+            m = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+            pb.prox_ffn_forward(p.h, p.t_x[t], 1, k1, k2, y)
+            pb.prox_ffn_last_mask(p.h, 1, k2, m)
+            torch.cuda.synchronize()
+            outs.append((y.cpu().numpy()[0], m.cpu().numpy()[0].astype(np.int64)))
+        pb.prox_ffn_set_fused(p.h, 1)
+        idx, score, sel_ref, thr = p.oracle_stage1(t, k1, k2)
+        for yv, mv in outs:
+            check_mask(mv, score, sel_ref, thr, k2, p.F)
+            y_ref, _ = po.stage2(p.x[t], mv, p.wg, p.wu, p.wd)
+            assert check_y(yv, y_ref) < 1e-4
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("k1,k2", [(512, 1536), (1, 1), (512, 1), (17, 1535), (300, 768), (16, 148), (33, 149)])
+def test_fused_edge_budgets(pb, toy, k1, k2):
+    wl, p = toy
+    p.quantize(4, 128)
+    for t in (2, 7):
+        _forward_check(pb, p, t, k1, k2)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+def test_fused_all_zero_input(pb, toy):
+    """x = 0: every score ties at 0; the mask must be the first k2 channels and y = 0."""
+    wl, p = toy
+    p.quantize(4, 0)
+    k1, k2 = wl.points[50]
+    xz = torch.zeros(1, p.D, dtype=torch.bfloat16, device="cuda")
+    y = p.y_empty()
+    m = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+    pb.prox_ffn_forward(p.h, xz, 1, k1, k2, y)
+    pb.prox_ffn_last_mask(p.h, 1, k2, m)
+    torch.cuda.synchronize()
+    assert np.array_equal(m.cpu().numpy()[0], np.arange(k2))
+    assert float(y.abs().max()) == 0.0
 
 
 # --------------------------------------------------------- threshold variant

@@ -34,12 +34,16 @@ def _run(pb, name, n_tok, cases, batches=(1,)):
                     xb = p.t_x[t0:t0 + B]
                     pb.prox_stage1_mask(p.h, xb, B, k1, k2, sel)
                     pb.prox_ffn_forward(p.h, xb, B, k1, k2, y)
+                    used = torch.empty_like(sel)           # the mask the forward call itself built
+                    pb.prox_ffn_last_mask(p.h, B, k2, used)
                     torch.cuda.synchronize()
-                    sel_np, y_np = sel.cpu().numpy().astype(np.int64), y.cpu().numpy()
+                    sel_np, used_np, y_np = (sel.cpu().numpy().astype(np.int64),
+                                             used.cpu().numpy().astype(np.int64), y.cpu().numpy())
                     for b in range(B):
                         idx, score, sel_ref, thr = p.oracle_stage1(t0 + b, k1, k2)
                         check_mask(sel_np[b], score, sel_ref, thr, k2, p.F)
-                        y_ref, _ = po.stage2(p.x[t0 + b], sel_np[b], p.wg, p.wu, p.wd)
+                        check_mask(used_np[b], score, sel_ref, thr, k2, p.F)
+                        y_ref, _ = po.stage2(p.x[t0 + b], used_np[b], p.wg, p.wu, p.wd)
                         check_y(y_np[b], y_ref)
                     if B == 1:
                         # Stage 2 alone, fed the oracle's own mask
@@ -76,8 +80,8 @@ def test_llama3_70b_s1_sweep(pb):
         for k1, k2 in wl.extra["s1_sweep"][::3]:
             y = p.y_empty()
             sel = torch.empty(1, k2, dtype=torch.int32, device="cuda")
-            pb.prox_stage1_mask(p.h, p.t_x[0], 1, k1, k2, sel)
             pb.prox_ffn_forward(p.h, p.t_x[0], 1, k1, k2, y)
+            pb.prox_ffn_last_mask(p.h, 1, k2, sel)
             torch.cuda.synchronize()
             sel_np = sel.cpu().numpy()[0].astype(np.int64)
             idx, score, sel_ref, thr = p.oracle_stage1(0, k1, k2)
