@@ -131,6 +131,15 @@ prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
  * slots, registers per thread, static shared bytes, co-resident blocks per SM}. */
 prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* info_host);
 
+/* Debug aid: with on != 0 every block of the persistent kernel records time
+ * stamps (nanoseconds of the GPU's global timer) per call: slots 0..9 mark the
+ * ends of set-up, input mask, proxy GEMV, grid barrier, channel mask, (unused),
+ * gate/up + down, partial-y exchange and finalize; slots 10..31 are finer marks
+ * inside those phases.  If stamps_host is given, the stamps of the last call are
+ * copied to it as [min(max_blocks, SM count)][32] uint64 (synchronises).
+ * on = 0 frees the buffer. */
+prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int max_blocks);
+
 /* Copy the channel mask of the most recent prox_ffn_forward call (top-k rule)
  * into sel_dev, dev int32 [B, k2], ascending per token.  Enqueued on stream. */
 prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev, void* stream);

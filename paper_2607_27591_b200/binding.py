@@ -63,6 +63,7 @@ _SIGS = {
     "prox_last_device_status": [_vp, C.POINTER(C.c_int32), _vp],
     "prox_launch_count": [_vp, C.POINTER(C.c_int64)],
     "prox_ffn_set_fused": [_vp, _i],
+    "prox_fused_trace": [_vp, _i, _vp, _i],
     "prox_fused_kernel_info": [_vp, _i, _i, C.POINTER(C.c_int32)],
     "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
     "prox_profile_enable": [_vp, _i],
@@ -149,6 +150,10 @@ def prox_fused_kernel_info(handle: int, k1: int, k2: int) -> dict:
     _check(_lib.prox_fused_kernel_info(handle, k1, k2, info), "prox_fused_kernel_info")
     keys = ("usable", "grid", "ksplit", "smem_bytes", "ring_slots", "registers", "static_smem", "blocks_per_sm")
     return dict(zip(keys, list(info)))
+
+
+def prox_fused_trace(handle: int, on: int, stamps_host=None, max_blocks: int = 0) -> None:
+    _check(_lib.prox_fused_trace(handle, int(on), _ptr(stamps_host), max_blocks), "prox_fused_trace")
 
 
 def prox_ffn_last_mask(handle: int, B: int, k2: int, sel, stream=None) -> None:

@@ -47,10 +47,11 @@ struct prox_ffn {
   int* dev_status;
   unsigned long long* counters;  // [0] tokens, [1] kept inputs, [2] kept channels
   unsigned* syncbuf;        // fused kernel: [0..2047] score histogram, [2048] barrier count,
-                            // [2049] barrier generation, [2050] finish ticket
+                            // (64-bit, [2048..2049]), [2050] finish ticket
   int smem_optin;           // largest dynamic shared memory a block may ask for
   int coop;                 // device supports cooperative launch
   int use_fused;            // batch-1 forward runs as one persistent kernel
+  unsigned long long* trace;  // optional phase time stamps of the persistent kernel (debug)
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -237,14 +238,16 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   if (!h->use_fused || !h->coop) return pl;
   const int G = h->sm_count;
-  const size_t fixed = ((sizeof(FusedSmem) + 127) & ~size_t(127)) + (size_t)4 * D;
+  const size_t fixed = ((sizeof(FusedSmem) + 127) & ~size_t(127)) + (size_t)8 * D;   // + x bf16, idx, x fp32
   if ((size_t)h->smem_optin < fixed + (size_t)6 * D + 16384) return pl;
   pl.big_bytes = (int)(((size_t)h->smem_optin - fixed) & ~size_t(127));
   pl.nslots = pl.big_bytes / (2 * D);
   if (pl.nslots > kMaxSlots) pl.nslots = kMaxSlots;
   if (pl.nslots < 3) return pl;
-  if (pl.big_bytes < kFusedConsumerWarps * 2 * 512) return pl;          // one row per warp buffer
-  if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;  // reduction scratch
+  const int scb = 2 * ch_per_chunk(h->bits) * 2 * 32;                    // one (group, strip) scale block
+  if (pl.big_bytes < kFusedConsumerWarps * (kScaleGroupsPerWarp * scb + kProxyRowsInFlight * 512)) return pl;   // proxy row buffers
+  if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;      // reduction scratch
+  if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
   if ((k2 + G - 1) / G > kMySelCap) return pl;
   pl.nstrips = nstrips_for(F, h->bits);
   // row split: fill the grid evenly (items = strips * ksplit run in rounds of G blocks)
@@ -260,17 +263,16 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   }
   pl.ksplit = best;
   pl.grid = G;
-  pl.xch = (D / 8 + kFusedConsumers - 1) / kFusedConsumers;
-  pl.xch = pl.xch <= 1 ? 1 : (pl.xch == 2 ? 2 : 4);
+  pl.xch = D <= 4096 ? 4 : (D <= 8192 ? 2 : 1);          // warp groups of the down projection
   pl.smem = fixed + (size_t)pl.big_bytes;
   pl.ok = true;
   return pl;
 }
 
-template <int BITS, int XCH>
+template <int BITS, int NG>
 cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
   static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
-  auto kern = prox_fused_kernel<BITS, XCH>;
+  auto kern = prox_fused_kernel<BITS, NG>;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
@@ -302,18 +304,19 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.nstrips = pl.nstrips; prm.ksplit = pl.ksplit;
   prm.part = h->part; prm.ticket = h->ticket; prm.scores = h->scores; prm.ghist = h->syncbuf;
   prm.sel_out = sel_out; prm.yacc = h->yacc;
-  prm.bar_count = h->syncbuf + 2048; prm.bar_gen = h->syncbuf + 2049; prm.done_ticket = h->syncbuf + 2050;
+  prm.bar_count = reinterpret_cast<unsigned long long*>(h->syncbuf + 2048); prm.done_ticket = h->syncbuf + 2050;
   prm.status = h->dev_status;
   prm.big_bytes = pl.big_bytes; prm.nslots = pl.nslots;
+  prm.trace = h->trace;
   cudaError_t e;
   {
     LaunchScope ls(h, kKFused, st);
     if (h->bits == 4) {
-      e = pl.xch == 1 ? launch_fused_t<4, 1>(pl, prm, st)
-        : pl.xch == 2 ? launch_fused_t<4, 2>(pl, prm, st) : launch_fused_t<4, 4>(pl, prm, st);
+      e = pl.xch == 4 ? launch_fused_t<4, 4>(pl, prm, st)
+        : pl.xch == 2 ? launch_fused_t<4, 2>(pl, prm, st) : launch_fused_t<4, 1>(pl, prm, st);
     } else {
-      e = pl.xch == 1 ? launch_fused_t<8, 1>(pl, prm, st)
-        : pl.xch == 2 ? launch_fused_t<8, 2>(pl, prm, st) : launch_fused_t<8, 4>(pl, prm, st);
+      e = pl.xch == 4 ? launch_fused_t<8, 4>(pl, prm, st)
+        : pl.xch == 2 ? launch_fused_t<8, 2>(pl, prm, st) : launch_fused_t<8, 1>(pl, prm, st);
     }
   }
   CK(e);
@@ -390,7 +393,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   free_packed(h);
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
-  cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf);
+  cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -505,6 +508,22 @@ prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* inf
   CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kFusedThreads, pl.smem));
   info[1] = pl.grid; info[2] = pl.ksplit; info[3] = (int)pl.smem; info[4] = pl.nslots;
   info[5] = fa.numRegs; info[6] = (int)fa.sharedSizeBytes; info[7] = nb;
+  return PROX_OK;
+}
+
+prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int max_blocks) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  const int G = h->sm_count;
+  if (on && !h->trace) {
+    CK(dev_alloc(&h->trace, (size_t)G * 32));
+    CK(cudaMemset(h->trace, 0, (size_t)G * 32 * sizeof(unsigned long long)));
+  }
+  if (stamps_host && h->trace) {
+    CK(cudaDeviceSynchronize());
+    const int n = max_blocks < G ? max_blocks : G;
+    CK(cudaMemcpy(stamps_host, h->trace, (size_t)n * 32 * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  }
+  if (!on && h->trace) { cudaFree(h->trace); h->trace = nullptr; }
   return PROX_OK;
 }
 

@@ -327,6 +327,35 @@ __device__ __forceinline__ void proxy_accumulate(const uint4& v, float xv, float
   }
 }
 
+// Variant that forms the exact integer code q = n - 8 with full-rate
+// instructions only.  A 4-bit code sitting at bit 4m (m <= 4) of a word, OR-ed
+// into the mantissa of 2^(23-4m), is the float 2^(23-4m) + n; one LOP3 isolates
+// it, one FADD removes 2^(23-4m) + 8, one FFMA accumulates q * x (exact product,
+// nothing to correct later).  The three codes above bit 19 are reached through
+// one shift of the word by 12.  On this GPU shifts, byte permutes and packed
+// half arithmetic issue at half the rate of LOP3 / FADD / FFMA.
+template <int BITS>
+__device__ __forceinline__ void proxy_accumulate_exact(const uint4& v, float xv, float* acc) {
+  if (BITS == 4) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t hi = w[q] >> 12;
+#pragma unroll
+      for (int m = 0; m < 8; ++m) {
+        const int pos = (m < 5) ? m : (m - 3);                  // code position inside w or inside hi
+        const uint32_t src = (m < 5) ? w[q] : hi;
+        const uint32_t magic = (uint32_t)(150 - 4 * pos) << 23;  // 2^(23 - 4 pos)
+        const float off = (float)(1u << (23 - 4 * pos)) + 8.0f;
+        const float f = __uint_as_float((src & (0xFu << (4 * pos))) | magic) - off;
+        acc[q * 8 + m] = fmaf(f, xv, acc[q * 8 + m]);
+      }
+    }
+  } else {
+    proxy_accumulate<8>(v, xv, acc);
+  }
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(kProxyThreads)
 proxy_gemv_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
