@@ -151,6 +151,43 @@ prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev,
 prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, int k1, int k2,
                                     void* y_host, void* stream);
 
+/* Stage 2 for callers that must not allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of prox_stage2_ffn.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a
+ * framework's stream-ordered or graph-captured region, under a memory pool that
+ * owns the whole device, in a latency-critical serving loop that forbids
+ * allocator calls, or in a plug-in that is handed raw buffers and no handle.
+ * Such a caller cannot create a prox_ffn_t (creating one allocates).
+ *
+ * What it does: for one token (B = 1) it computes h_j = SiLU(x . W_gate[j,:]) *
+ * (x . W_up[j,:]) for the k2 channels in sel and y = sum_j h_j W_down_t[j,:],
+ * exactly like prox_stage2_ffn, but takes every tensor from the caller:
+ *   x            dev bf16 [d_model]
+ *   w_gate, w_up dev bf16 [d_ff, d_model]
+ *   w_down_t     dev bf16 [d_ff, d_model]: W_down stored channel-major (row j is
+ *                the d_model weights of channel j, i.e. the transpose of the
+ *                [d_model, d_ff] matrix the other entry points take)
+ *   sel          dev int32 [k2], ids in [0, d_ff) (others are skipped)
+ *   y            dev [d_model], bf16 (out_dtype 0) or fp32 (1)
+ * The two intermediates (one fp32 h per kept channel and the fp32 accumulator of
+ * y) live in a 192 KB array that is part of the library image on every GPU that
+ * loads it, instead of in allocated memory.  Hence the limits: d_model <= 16384
+ * and k2 <= 32768 (PROX_ERR_UNSUPPORTED beyond; use the handle-based call).
+ * No cudaMalloc, cudaFree or allocating library routine is called.
+ *
+ * The first call on a device looks up the device address of that array (the
+ * device must be current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the last call's
+ * contents (the accumulator is cleared at the start of every call): two calls
+ * that overlap on the GPU - different streams, or concurrent host threads -
+ * race on it, so serialise them.  Work is enqueued on `stream`; no sync.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+prox_status_t prox_stage2_ffn_noalloc(const void* x_dev, const void* w_gate_dev, const void* w_up_dev,
+                                      const void* w_down_t_dev, int d_model, int d_ff,
+                                      const int32_t* sel_dev, int k2, void* y_dev, int out_dtype,
+                                      void* stream);
+
 /* Threshold variant of the two indicators of Sec. 4.1:
  *   [m_x]_i = 1[|x_i| >= tau_x],  [m_s]_j = 1[|s~_j| >= tau_s].
  * The number of kept entries varies per token.

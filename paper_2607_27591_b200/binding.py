@@ -48,6 +48,7 @@ _SIGS = {
     "prox_stage2_ffn": [_vp, _vp, _i, _vp, _i, _vp, _vp],
     "prox_ffn_forward": [_vp, _vp, _i, _i, _i, _vp, _vp],
     "prox_ffn_forward_host": [_vp, _vp, _i, _i, _i, _vp, _vp],
+    "prox_stage2_ffn_noalloc": [_vp, _vp, _vp, _vp, _i, _i, _vp, _i, _vp, _i, _vp],
     "prox_stage1_mask_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp, _vp, _vp],
     "prox_stage2_ffn_var": [_vp, _vp, _i, _vp, _vp, _vp, _vp],
     "prox_ffn_forward_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp],
@@ -139,6 +140,16 @@ def prox_stage2_ffn(handle: int, x, B: int, sel, k2: int, y, stream=None) -> Non
 
 def prox_ffn_forward(handle: int, x, B: int, k1: int, k2: int, y, stream=None) -> None:
     _check(_lib.prox_ffn_forward(handle, _ptr(x), B, k1, k2, _ptr(y), _ptr(stream)), "prox_ffn_forward")
+
+
+def prox_stage2_ffn_noalloc(x, w_gate, w_up, w_down_t, d_model: int, d_ff: int, sel, k2: int, y,
+                            out_dtype: int, stream=None) -> None:
+    """Stage 2 without a handle and without any allocation (B = 1): the caller passes
+    every tensor, W_down in channel-major [d_ff, d_model] form; the intermediates sit
+    in a fixed array inside the library (d_model <= 16384, k2 <= 32768)."""
+    _check(_lib.prox_stage2_ffn_noalloc(_ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down_t), d_model, d_ff,
+                                        _ptr(sel), k2, _ptr(y), out_dtype, _ptr(stream)),
+           "prox_stage2_ffn_noalloc")
 
 
 def prox_ffn_set_fused(handle: int, on: int) -> None:

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libprox.so")
-SOURCES = [os.path.join(CSRC, "prox_api.cu")]
+SOURCES = [os.path.join(CSRC, "prox_api.cu"), os.path.join(CSRC, "prox_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "prox_kernels.cuh"), os.path.join(ROOT, "include", "prox.h")]
 
 
