@@ -54,6 +54,21 @@ def parse():
     return ap.parse_args()
 
 
+def ncu_traffic():
+    """DRAM bytes per launch of the fused kernel from the committed ncu summary (profiles/), or None."""
+    path = os.path.join(ROOT, "profiles", "prox_fused_kernel_qwen3_8b_ncu_full.md")
+    try:
+        for line in open(path):
+            if line.startswith("| **traffic"):
+                cells = [c.strip(" *") for c in line.strip().strip("|").split("|")]
+                vals = [float(c.split()[0]) for c in cells[1:] if c and c.split()[0].replace(".", "").isdigit()]
+                if vals:
+                    return sum(vals) / len(vals) * 1e6
+    except OSError:
+        pass
+    return None
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -357,7 +372,8 @@ def run_prox(args):
     if dom:
         ach = per_kernel[dom]["gbs"]
         roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s",
-                "frac": ach / peak, "peak_kind": peak_kind, "traffic": None,
+                "frac": ach / peak, "peak_kind": peak_kind,
+                "traffic": ncu_traffic() if dom == "prox_fused" else None,
                 "bytes_per_launch": kernel_bytes.get(dom)}
 
     cpu = None
