@@ -200,6 +200,26 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------- multi-rank reduction
+def max_over_ranks(values, device=None):
+    """Every rank passes its own timings; all ranks get the element-wise maximum.
+    With one process (no process group) the values come back unchanged.  The path
+    has no data-path collective: ranks are independent replicas, and this MAX of
+    a few timing scalars is the only exchange."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_us_per_call(ms_max, world, steps, calls_per_step):
+    """Whole-job figure: all ranks together made world*steps*calls_per_step calls
+    in ms_max (the slowest rank's time)."""
+    return ms_max * 1e3 / (world * steps * calls_per_step)
+
+
 # ------------------------------------------------------------------ GPU leg
 def run_prox(args):
     import torch
@@ -322,38 +342,60 @@ def run_prox(args):
         sync_all()
         e2e_s = time.perf_counter() - t0
 
+        def timed_graph(fn, reps=5):
+            """Capture fn() (one pass over the replicas) in a graph; µs per replay, or None."""
+            try:
+                fn(); stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    fn()
+                for _ in range(3):
+                    g.replay()
+                stream.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(reps):
+                    g.replay()
+                b.record(stream)
+                stream.synchronize()
+                return a.elapsed_time(b) / reps * 1e3
+            except Exception as ex:                    # pragma: no cover
+                sys.stderr.write(f"side measurement failed: {ex}\n")
+                return None
+
         # dense bf16 cuBLAS FFN on the same replicas (context)
         def dense_step():
             for t in range(T):
                 wg, wu, wd = weights[t % R]
                 g = torch.mv(wg, x[t]); u = torch.mv(wu, x[t])
                 torch.mv(wd, torch.nn.functional.silu(g) * u, out=y[t])
-        dense_us = None
-        try:
-            dense_step(); stream.synchronize()
-            dg = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(dg, stream=stream):
-                dense_step()
-            for _ in range(3):
-                dg.replay()
-            stream.synchronize()
-            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            d0.record(stream)
-            for _ in range(5):
-                dg.replay()
-            d1.record(stream)
-            stream.synchronize()
-            dense_us = d0.elapsed_time(d1) / (5 * T) * 1e3
-        except Exception as ex:                        # pragma: no cover
-            sys.stderr.write(f"dense comparison failed: {ex}\n")
+        dense_us = timed_graph(dense_step)
+        dense_us = dense_us / T if dense_us else None
 
-    tms = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(tms[0]), float(tms[1])
-    calls = world * args.steps * T
-    us_per_call = ms * 1e3 / calls
-    e2e_us = e2e_ms * 1e3 / (world * e2e_steps * T)
+        # batch 8 with per-token masks (union path) and dense cuBLAS at batch 8, same replicas
+        B8, calls8 = 8, 2 * R
+        x8 = x[:B8 * 8].reshape(8, B8, D)
+        y8 = torch.empty(8, B8, D, dtype=torch.bfloat16, device=dev)
+
+        def prox8_step():
+            cs = torch.cuda.current_stream().cuda_stream
+            for c in range(calls8):
+                pb.prox_ffn_forward(handles[c % R], x8[c % 8], B8, k1, k2, y8[c % 8], stream=cs)
+
+        def dense8_step():
+            for c in range(calls8):
+                wg, wu, wd = weights[c % R]
+                xb = x8[c % 8]
+                torch.matmul(torch.nn.functional.silu(xb @ wg.t()) * (xb @ wu.t()), wd.t(), out=y8[c % 8])
+        b8_us = timed_graph(prox8_step)
+        d8_us = timed_graph(dense8_step)
+        batch8 = {"batch": B8, "prox_us_per_call": b8_us / calls8 if b8_us else None,
+                  "dense_cublas_bf16_us_per_call": d8_us / calls8 if d8_us else None,
+                  "masks": "per token; weights read once for the union"}
+
+    ms, e2e_ms = max_over_ranks([ms, e2e_s * 1e3], dev)
+    us_per_call = whole_job_us_per_call(ms, world, args.steps, T)
+    e2e_us = whole_job_us_per_call(e2e_ms, world, e2e_steps, T)
 
     s1b, gub, dnb, actb = pb.prox_algorithmic_bytes(handles[0], k1, k2)
     bytes_call = s1b + gub + dnb + actb
@@ -402,6 +444,7 @@ def run_prox(args):
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": T * D * 2, "d2h_bytes_per_step": T * D * 2},
             "gpu_launches": int(round(launches_per_call * T * args.steps)),
             "dense_cublas_bf16_us_per_call": dense_us,
+            "batch8": batch8,
             "clocks": clocks,
         }
         print(json.dumps(out))

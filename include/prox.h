@@ -126,6 +126,13 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x_dev, int B, int k1, 
  * prox_last_device_status reports bit 4. */
 prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
 
+/* For B > 1 every token keeps its own masks (the paper covers B = 1 only), and the
+ * weights are read once per call for the UNION of the tokens' kept inputs and of
+ * their kept channels; a token contributes zero outside its own masks, so its
+ * result is the one it would get alone.  prox_ffn_set_union(h, 0) selects the
+ * older path that runs the single-token kernels once per token. */
+prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on);
+
 /* Launch plan of the persistent kernel for budgets (k1, k2), for diagnostics:
  * info[8] (host) = {usable, grid blocks, row split, dynamic shared bytes, ring
  * slots, registers per thread, static shared bytes, co-resident blocks per SM}. */
@@ -251,8 +258,8 @@ prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream
  * prox_profile_read synchronises those events, adds up launches and
  * milliseconds per kernel kind into counts[PROX_NUM_KERNEL_KINDS] and
  * ms[PROX_NUM_KERNEL_KINDS] (host arrays), and forgets them.  Kinds, in order:
- * input_select, proxy_gemv, channel_select, gateup, down, finalize, fused. */
-#define PROX_NUM_KERNEL_KINDS 7
+ * input_select, proxy_gemv, channel_select, gateup, down, finalize, fused, union. */
+#define PROX_NUM_KERNEL_KINDS 8
 prox_status_t prox_profile_enable(prox_ffn_t* h, int on);
 prox_status_t prox_profile_read(prox_ffn_t* h, int64_t* counts_host, double* ms_host);
 

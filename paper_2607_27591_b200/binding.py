@@ -64,6 +64,7 @@ _SIGS = {
     "prox_last_device_status": [_vp, C.POINTER(C.c_int32), _vp],
     "prox_launch_count": [_vp, C.POINTER(C.c_int64)],
     "prox_ffn_set_fused": [_vp, _i],
+    "prox_ffn_set_union": [_vp, _i],
     "prox_fused_trace": [_vp, _i, _vp, _i],
     "prox_fused_kernel_info": [_vp, _i, _i, C.POINTER(C.c_int32)],
     "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
@@ -154,6 +155,10 @@ def prox_stage2_ffn_noalloc(x, w_gate, w_up, w_down_t, d_model: int, d_ff: int, 
 
 def prox_ffn_set_fused(handle: int, on: int) -> None:
     _check(_lib.prox_ffn_set_fused(handle, int(on)), "prox_ffn_set_fused")
+
+
+def prox_ffn_set_union(handle: int, on: int) -> None:
+    _check(_lib.prox_ffn_set_union(handle, int(on)), "prox_ffn_set_union")
 
 
 def prox_fused_kernel_info(handle: int, k1: int, k2: int) -> dict:
@@ -248,7 +253,7 @@ def prox_launch_count(handle: int) -> int:
     return n.value
 
 
-KERNEL_KINDS = ("input_select", "proxy_gemv", "channel_select", "gateup", "down", "finalize", "prox_fused")
+KERNEL_KINDS = ("input_select", "proxy_gemv", "channel_select", "gateup", "down", "finalize", "prox_fused", "union")
 
 
 def prox_profile_enable(handle: int, on: int) -> None:

@@ -11,10 +11,11 @@
 
 #include "prox_kernels.cuh"
 #include "prox_fused.cuh"
+#include "prox_batch.cuh"
 
 using namespace prox;
 
-enum KernelKind { kKInput = 0, kKProxy, kKChannel, kKGateUp, kKDown, kKFinalize, kKFused };
+enum KernelKind { kKInput = 0, kKProxy, kKChannel, kKGateUp, kKDown, kKFinalize, kKFused, kKUnion };
 struct ProfRec { int kind; cudaEvent_t a, b; };
 
 struct prox_ffn {
@@ -51,7 +52,14 @@ struct prox_ffn {
   int smem_optin;           // largest dynamic shared memory a block may ask for
   int coop;                 // device supports cooperative launch
   int use_fused;            // batch-1 forward runs as one persistent kernel
+  int use_union;            // batch > 1 reads weights once for the union of the tokens' masks
   unsigned long long* trace;  // optional phase time stamps of the persistent kernel (debug)
+  // batch > 1: unions of the tokens' masks (allocated when max_batch > 1)
+  int* u_in; int* u_ch;     // [D], [F] ascending union lists
+  int* u_cnt;               // [0] union inputs, [1] union channels
+  float* xu;                // [D][8]  x of every token at a union input (0 if dropped)
+  float* member;            // [F][8]  1 / 0 membership of every token at a union channel
+  float* hb;                // [F][8]  h of every token at a union channel
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -225,6 +233,100 @@ prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, i
   return PROX_OK;
 }
 
+// ---- batch > 1: union path -----------------------------------------------------
+bool batch_path_ok(const prox_ffn* h, int B) {
+  if (B < 2 || !h->u_in) return false;
+  const size_t xs_bytes = (size_t)B * h->cfg.d_model * 2;
+  const size_t red_bytes = (size_t)4 * kBT * 128 * (h->bits == 4 ? 8 : 4) * sizeof(float);
+  const size_t ubits = (size_t)B * ((h->cfg.d_ff + 31) / 32) * 4;
+  const size_t lim = (size_t)h->smem_optin - 4096;
+  return xs_bytes <= lim && red_bytes <= lim && ubits <= lim;
+}
+
+prox_status_t launch_union(prox_ffn* h, const int* lists, int stride, const int* cnt, int k, int B, int n,
+                           const void* x, int* ulist, int* nu, float* val, cudaStream_t st) {
+  const size_t smem = (size_t)B * ((n + 31) / 32) * sizeof(unsigned);
+  static bool attr = false;
+  if (!attr) { CK(cudaFuncSetAttribute(union_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
+  {
+    LaunchScope ls(h, kKUnion, st);
+    union_kernel<<<1, 1024, smem, st>>>(lists, stride, cnt, k, B, n, static_cast<const uint16_t*>(x), ulist, nu, val,
+                                        h->dev_status);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
+prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int k2, int* sel, int sel_stride,
+                                  float* scores, cudaStream_t st) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  prox_status_t s;
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  if ((s = launch_union(h, h->idx_x, D, nullptr, k1, B, D, x, h->u_in, h->u_cnt, h->xu, st)) != PROX_OK) return s;
+  const int ns = nstrips_for(F, h->bits);
+  const int nval = 128 * (h->bits == 4 ? 8 : 4);
+  int ks = h->sm_count / ns;
+  if (ks < 1) ks = 1;
+  if (ks > 16) ks = 16;
+  while (ks > 1 && (size_t)ks * ns * kBT * nval > h->part_floats) --ks;
+  if ((size_t)ks * ns * kBT * nval > h->part_floats && ks > 1) return PROX_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)4 * kBT * nval * sizeof(float);
+  const int gshift = (h->group == D) ? 31 : 7;
+  dim3 grid(ns, ks);
+  {
+    LaunchScope ls(h, kKProxy, st);
+    if (h->bits == 4) {
+      static bool attr4 = false;
+      if (!attr4) { CK(cudaFuncSetAttribute(proxy_batch_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); attr4 = true; }
+      proxy_batch_kernel<4><<<grid, kPBThreads, smem, st>>>(h->P, h->S, h->u_in, h->u_cnt, h->xu, B, D, F, gshift,
+                                                           h->part, h->ticket, scores);
+    } else {
+      static bool attr8 = false;
+      if (!attr8) { CK(cudaFuncSetAttribute(proxy_batch_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); attr8 = true; }
+      proxy_batch_kernel<8><<<grid, kPBThreads, smem, st>>>(h->P, h->S, h->u_in, h->u_cnt, h->xu, B, D, F, gshift,
+                                                           h->part, h->ticket, scores);
+    }
+  }
+  CK(cudaGetLastError());
+  return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
+}
+
+prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* sel, int sel_stride, int k2,
+                                  void* y, cudaStream_t st) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  prox_status_t s;
+  if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK)
+    return s;
+  const size_t smem = (size_t)B * D * 2;
+  static bool attr = false;
+  if (!attr) { CK(cudaFuncSetAttribute(gateup_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
+  int blocks = (F + kGBThreads / 32 - 1) / (kGBThreads / 32);
+  const int cap = 8 * h->sm_count;
+  if (blocks > cap) blocks = cap;
+  {
+    LaunchScope ls(h, kKGateUp, st);
+    gateup_batch_kernel<<<blocks, kGBThreads, smem, st>>>(h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch,
+                                                         h->u_cnt + 1, h->member, D, F, h->hb);
+  }
+  CK(cudaGetLastError());
+  const int dtiles = (D + kDownThreads * 8 - 1) / (kDownThreads * 8);
+  int nsplit = (h->sm_count + dtiles - 1) / dtiles;
+  if (nsplit < 1) nsplit = 1;
+  dim3 g2(dtiles, nsplit);
+  {
+    LaunchScope ls(h, kKDown, st);
+    down_batch_kernel<<<g2, kDownThreads, 0, st>>>(h->wdt, h->hb, h->u_ch, h->u_cnt + 1, B, D, h->yacc);
+  }
+  CK(cudaGetLastError());
+  const int n = B * D;
+  {
+    LaunchScope ls(h, kKFinalize, st);
+    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, y, n, h->cfg.out_dtype);
+  }
+  CK(cudaGetLastError());
+  return PROX_OK;
+}
+
 // ---- fused persistent kernel (batch 1) ----------------------------------------
 struct FusedPlan {
   bool ok;
@@ -357,6 +459,10 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   const int D = cfg->d_model, F = cfg->d_ff, MB = cfg->max_batch;
   const int ns_max = nstrips_for(F, 8);            // 8-bit strips are narrower -> more of them
   h->part_floats = ((size_t)2 * h->sm_count + (size_t)MB * ns_max + 64) * 1024;
+  if (MB > 1) {                                    // union path: [row split][strip][8 tokens][1024]
+    const size_t need = ((size_t)h->sm_count + ns_max) * kBT * 1024;
+    if (need > h->part_floats) h->part_floats = need;
+  }
   prox_status_t st = PROX_OK;
   auto A = [&](cudaError_t er) { if (er != cudaSuccess && st == PROX_OK) st = map_cuda(er); };
   A(dev_alloc(&h->idx_x, (size_t)MB * D));
@@ -371,9 +477,15 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   A(dev_alloc(&h->dev_status, (size_t)1));
   A(dev_alloc(&h->counters, (size_t)4));
   A(dev_alloc(&h->syncbuf, (size_t)2048 + 64));
+  if (MB > 1) {
+    A(dev_alloc(&h->u_in, (size_t)D)); A(dev_alloc(&h->u_ch, (size_t)F)); A(dev_alloc(&h->u_cnt, (size_t)4));
+    A(dev_alloc(&h->xu, (size_t)D * kBT)); A(dev_alloc(&h->member, (size_t)F * kBT));
+    A(dev_alloc(&h->hb, (size_t)F * kBT));
+  }
   A(cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
   A(cudaDeviceGetAttribute(&h->coop, cudaDevAttrCooperativeLaunch, h->device));
   h->use_fused = 1;
+  h->use_union = 1;
   if (st == PROX_OK) A(cudaMemset(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned)));
   A(dev_alloc(reinterpret_cast<uint16_t**>(&h->x_stage), (size_t)MB * D));
   A(dev_alloc(reinterpret_cast<float**>(&h->y_stage), (size_t)MB * D));
@@ -394,6 +506,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
+  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -458,6 +571,7 @@ prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x, int B, int k1, int 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model;
   float* sc = scores ? scores : h->scores;
+  if (h->use_union && batch_path_ok(h, B)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st);
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, sc, st)) != PROX_OK) return s;
   return launch_channel_select(h, sc, B, k2, 0.f, 0, sel, k2, nullptr, st);
@@ -470,6 +584,8 @@ prox_status_t prox_stage2_ffn(prox_ffn_t* h, const void* x, int B, const int32_t
   if (!sel || !y || !aligned16(y)) return PROX_ERR_INVALID_ARG;
   if (k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
   if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  if (h->use_union && batch_path_ok(h, B))
+    return launch_stage2_batch(h, x, B, sel, k2, k2, y, static_cast<cudaStream_t>(stream));
   return launch_stage2(h, x, B, sel, k2, nullptr, k2, y, static_cast<cudaStream_t>(stream));
 }
 
@@ -484,6 +600,10 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
   if (B == 1) {
     const FusedPlan pl = plan_fused(h, k1, k2);
     if (pl.ok) return launch_fused(h, pl, x, k1, k2, y, h->sel, st);
+  }
+  if (h->use_union && batch_path_ok(h, B)) {
+    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st)) != PROX_OK) return s;
+    return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st);
   }
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
@@ -530,6 +650,12 @@ prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int
 prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on) {
   if (!h) return PROX_ERR_INVALID_ARG;
   h->use_fused = on != 0;
+  return PROX_OK;
+}
+
+prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  h->use_union = on != 0;
   return PROX_OK;
 }
 

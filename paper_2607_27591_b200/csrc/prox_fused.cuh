@@ -149,6 +149,15 @@ __device__ __forceinline__ bool slot_wait(uint32_t bar, volatile unsigned* seen,
   return true;
 }
 
+// Exclusive prefix over the lanes of a warp of popc(m8), m8 an 8-bit mask per
+// lane: eight ballots instead of a five-step shuffle scan (shuffles are slow here).
+__device__ __forceinline__ unsigned lane_prefix8(unsigned m8, unsigned lt_mask) {
+  unsigned pre = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) pre += __popc(__ballot_sync(0xffffffffu, (m8 >> e) & 1u) & lt_mask);
+  return pre;
+}
+
 // k-th largest bin of hist[0..NBINS) counted from the top, with two block
 // barriers: warps scan their bins with shuffles, every thread then adds up the
 // totals of the warps in front of it.  Result in res[0] (bin), res[1] (above).
@@ -332,61 +341,52 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       quota = (unsigned)k1 - above1 - above2;      // ties at T to accept, lowest index first
       PROX_TRACE(13);
     }
-    // per-chunk counts (kept: key > T, tie: key == T), then ordered compaction
-    unsigned* ccnt = sm.hist;                              // reuse: [nchk] packed counts, then bases
-    for (int q = warp; q < nchk; q += kFusedWarps) {
-      const int v = q * 32 + lane;
-      unsigned cg = 0, ce = 0;
-      if (v < nvec) {
-        const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
-        const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+    // Ordered compaction.  A warp keeps the kept/tie masks of its chunks in
+    // registers, counts them with one warp reduction and prefixes them with ballots.
+    unsigned* ccnt = sm.hist;                              // reuse: [1024 + q] packed counts of chunk q
+    constexpr int MAXC = 4;                                // chunks per warp (64 chunks / 20 warps)
+    unsigned gmv[MAXC], emv[MAXC], pgv[MAXC], pev[MAXC];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const unsigned k0 = w[e] & 0x7fffu, k1b = (w[e] >> 16) & 0x7fffu;
-          cg += (k1 >= D || k0 > T) ? 1u : 0u;  cg += (k1 >= D || k1b > T) ? 1u : 0u;
-          ce += (k1 < D && k0 == T) ? 1u : 0u;  ce += (k1 < D && k1b == T) ? 1u : 0u;
+    for (int sidx = 0; sidx < MAXC; ++sidx) {
+      const int q = warp + sidx * kFusedWarps;
+      gmv[sidx] = emv[sidx] = pgv[sidx] = pev[sidx] = 0;
+      if (q < nchk) {                                      // warp-uniform
+        const int v = q * 32 + lane;
+        unsigned gm = 0, em = 0;
+        if (v < nvec) {
+          const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
+          const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const unsigned key = (w[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
+            gm |= ((k1 >= D || key > T) ? 1u : 0u) << e;
+            em |= ((k1 < D && key == T) ? 1u : 0u) << e;
+          }
         }
+        gmv[sidx] = gm; emv[sidx] = em;
+        pgv[sidx] = lane_prefix8(gm, lt_mask);
+        pev[sidx] = lane_prefix8(em, lt_mask);
+        const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(gm) | ((unsigned)__popc(em) << 16));
+        if (lane == 0) ccnt[1024 + q] = tot;
       }
-      unsigned pk = cg | (ce << 16);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) pk += __shfl_xor_sync(0xffffffffu, pk, o);
-      if (lane == 0) ccnt[1024 + q] = pk;
     }
     __syncthreads();
     PROX_TRACE(14);
-    for (int q = warp; q < nchk; q += kFusedWarps) {
-      // base of this chunk = counts of the chunks in front of it (<= 64 of them)
-      unsigned bsum = 0;
-      for (int j = lane; j < q; j += 32) bsum += ccnt[1024 + j];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) bsum += __shfl_xor_sync(0xffffffffu, bsum, o);
-      const int v = q * 32 + lane;
-      uint32_t w[4] = {0, 0, 0, 0};
-      unsigned gm = 0, em = 0;
-      if (v < nvec) {
-        const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
-        w[0] = kv.x; w[1] = kv.y; w[2] = kv.z; w[3] = kv.w;
+    for (int sidx = 0; sidx < MAXC; ++sidx) {
+      const int q = warp + sidx * kFusedWarps;
+      if (q < nchk) {
+        unsigned bsum = 0;                                 // counts of the chunks in front (<= 64)
+        for (int j = lane; j < q; j += 32) bsum += ccnt[1024 + j];
+        bsum = __reduce_add_sync(0xffffffffu, bsum);
+        unsigned rg = (bsum & 0xffffu) + pgv[sidx], re = (bsum >> 16) + pev[sidx];
+        const int v = q * 32 + lane;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const unsigned key = (w[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
-          gm |= ((k1 >= D || key > T) ? 1u : 0u) << e;
-          em |= ((k1 < D && key == T) ? 1u : 0u) << e;
+          const bool gt = (gmv[sidx] >> e) & 1u, eq = (emv[sidx] >> e) & 1u;
+          if (gt || (eq && re < quota)) idx16[rg + min(re, quota)] = (uint16_t)(v * 8 + e);
+          rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
         }
-      }
-      const unsigned mine = (unsigned)__popc(gm) | ((unsigned)__popc(em) << 16);
-      unsigned inc = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += t;
-      }
-      const unsigned ex = bsum + inc - mine;
-      unsigned rg = ex & 0xffffu, re = ex >> 16;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const bool gt = (gm >> e) & 1u, eq = (em >> e) & 1u;
-        if (gt || (eq && re < quota)) idx16[rg + min(re, quota)] = (uint16_t)(v * 8 + e);
-        rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
       }
     }
     __syncthreads();
@@ -618,23 +618,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     const unsigned b1 = sm.res[0];
     unsigned kk = (unsigned)k2 - sm.res[1];
     PROX_TRACE(17);
-    // scores -> shared memory; members of the threshold bin become candidates
-    for (int i0 = tid * 4; i0 < F; i0 += NT * 4 * 4) {        // F % 4 == 0; loads first, then the stores
-      uint4 kv[4];
+    // scores -> shared memory, 256 channels per warp step (8 keys per lane);
+    // members of the threshold bin become candidates; channels above it are
+    // counted per chunk right away (they are selected whatever the exact threshold).
+    unsigned* ccnt = sm.hist;                              // [q] kept, [1024 + q] ties, per 256-channel chunk
+    const int nchk = (F + 255) / 256;                      // <= 256
+    __syncthreads();                                       // find_kth_fast is done with sm.hist
+    for (int q = warp; q < nchk; q += kFusedWarps) {
+      const int base = q * 256 + lane * 8;
+      uint4 kv[2];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * NT * 4;
-        kv[u] = (i < F) ? __ldcg(reinterpret_cast<const uint4*>(gkey + i)) : make_uint4(0, 0, 0, 0);
-      }
+      for (int hh = 0; hh < 2; ++hh)
+        kv[hh] = (base + hh * 4 < F) ? __ldcg(reinterpret_cast<const uint4*>(gkey + base + hh * 4)) : make_uint4(0, 0, 0, 0);
+      unsigned hi = 0;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * NT * 4;
+      for (int hh = 0; hh < 2; ++hh) {
+        const int i = base + hh * 4;
         if (i < F) {
-          if (in_smem) *reinterpret_cast<uint4*>(skey + i) = kv[u];
-          const unsigned kk4[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+          if (in_smem) *reinterpret_cast<uint4*>(skey + i) = kv[hh];
+          const unsigned kk4[4] = {kv[hh].x, kv[hh].y, kv[hh].z, kv[hh].w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            if ((kk4[e] >> 20) == b1) {
+            const unsigned bin = kk4[e] >> 20;
+            hi += (bin > b1) ? 1u : 0u;
+            if (bin == b1) {
               const unsigned slot = atomicAdd(&sm.ncand, 1u);
               if (slot < (unsigned)kCandCap) {
                 cand_key[slot] = kk4[e]; cand_idx[slot] = i + e;
@@ -644,6 +651,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           }
         }
       }
+      hi = __reduce_add_sync(0xffffffffu, hi);
+      if (lane == 0) { ccnt[q] = hi; ccnt[1024 + q] = 0; }
     }
     __syncthreads();
     const unsigned ncand = sm.ncand;
@@ -706,21 +715,29 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       }
       T = prefix; quota = kk;
     }
-    // Ordered compaction, 256 channels per warp step (8 keys per lane).  Only
-    // the chunks whose slice of the ascending list meets [R0, R1) write anything.
-    {
-      const int nchk = (F + 255) / 256;                    // <= 256
-      unsigned* ccnt = sm.hist;                             // [nchk] kept counts, [1024 + nchk] tie counts
-      auto load8 = [&](int base, unsigned* key) {
+    // Per-chunk counts: the channels above the threshold bin are counted already;
+    // add the candidates that made it (key > T) and note the ties (key == T).
+    bool counted = false;
+    if (have_T && ncand <= (unsigned)kCandCap) {
+      for (unsigned c = tid; c < ncand; c += NT) {
+        const unsigned key = cand_key[c];
+        const int chunk = cand_idx[c] >> 8;
+        if (key > T) atomicAdd(&ccnt[chunk], 1u);
+        else if (key == T) atomicAdd(&ccnt[1024 + chunk], 1u);
+      }
+      counted = true;
+    }
+    auto load8 = [&](int base, unsigned* key) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int i = base + h * 4;
-          uint4 kv = make_uint4(0, 0, 0, 0);
-          if (i < F) kv = in_smem ? *reinterpret_cast<const uint4*>(skey + i)
-                                  : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
-          key[h * 4 + 0] = kv.x; key[h * 4 + 1] = kv.y; key[h * 4 + 2] = kv.z; key[h * 4 + 3] = kv.w;
-        }
-      };
+      for (int hh = 0; hh < 2; ++hh) {
+        const int i = base + hh * 4;
+        uint4 kv = make_uint4(0, 0, 0, 0);
+        if (i < F) kv = in_smem ? *reinterpret_cast<const uint4*>(skey + i)
+                                : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
+        key[hh * 4 + 0] = kv.x; key[hh * 4 + 1] = kv.y; key[hh * 4 + 2] = kv.z; key[hh * 4 + 3] = kv.w;
+      }
+    };
+    if (!counted) {                                        // rare path: count every chunk from the keys
       for (int q = warp; q < nchk; q += kFusedWarps) {
         const int base = q * 256 + lane * 8;
         unsigned key[8];
@@ -732,56 +749,45 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           cg += (in && key[e] > T) ? 1u : 0u;
           ce += (in && key[e] == T) ? 1u : 0u;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          cg += __shfl_xor_sync(0xffffffffu, cg, o);
-          ce += __shfl_xor_sync(0xffffffffu, ce, o);
-        }
+        cg = __reduce_add_sync(0xffffffffu, cg);
+        ce = __reduce_add_sync(0xffffffffu, ce);
         if (lane == 0) { ccnt[q] = cg; ccnt[1024 + q] = ce; }
       }
-      __syncthreads();
-      PROX_TRACE(21);
-      for (int q = warp; q < nchk; q += kFusedWarps) {
-        unsigned bg = 0, be = 0;
-        for (int j = lane; j < q; j += 32) { bg += ccnt[j]; be += ccnt[1024 + j]; }
+    }
+    __syncthreads();
+    PROX_TRACE(21);
+    // Ordered compaction: only the chunks whose slice of the ascending list meets
+    // [R0, R1) write anything.
+    for (int q = warp; q < nchk; q += kFusedWarps) {
+      unsigned bg = 0, be = 0;
+      for (int j = lane; j < q; j += 32) { bg += ccnt[j]; be += ccnt[1024 + j]; }
+      bg = __reduce_add_sync(0xffffffffu, bg);
+      be = __reduce_add_sync(0xffffffffu, be);
+      const unsigned cgq = ccnt[q], ceq = ccnt[1024 + q];
+      const int first = (int)(bg + min(be, quota)), end = (int)(bg + cgq + min(be + ceq, quota));
+      if (first >= R1 || end <= R0) continue;              // warp-uniform
+      const int base = q * 256 + lane * 8;
+      unsigned key[8];
+      load8(base, key);
+      unsigned gm = 0, em = 0;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          bg += __shfl_xor_sync(0xffffffffu, bg, o);
-          be += __shfl_xor_sync(0xffffffffu, be, o);
-        }
-        const unsigned cgq = ccnt[q], ceq = ccnt[1024 + q];
-        const int first = (int)(bg + min(be, quota)), end = (int)(bg + cgq + min(be + ceq, quota));
-        if (first >= R1 || end <= R0) continue;            // warp-uniform
-        const int base = q * 256 + lane * 8;
-        unsigned key[8];
-        load8(base, key);
-        unsigned gm = 0, em = 0;
+      for (int e = 0; e < 8; ++e) {
+        const bool in = base + e < F;
+        gm |= ((in && key[e] > T) ? 1u : 0u) << e;
+        em |= ((in && key[e] == T) ? 1u : 0u) << e;
+      }
+      unsigned rg = bg + lane_prefix8(gm, lt_mask), re = be + lane_prefix8(em, lt_mask);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const bool in = base + e < F;
-          gm |= ((in && key[e] > T) ? 1u : 0u) << e;
-          em |= ((in && key[e] == T) ? 1u : 0u) << e;
-        }
-        unsigned ig = (unsigned)__popc(gm), ie = (unsigned)__popc(em);
-        const unsigned mg = ig, me = ie;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const unsigned tg = __shfl_up_sync(0xffffffffu, ig, o), te = __shfl_up_sync(0xffffffffu, ie, o);
-          if (lane >= o) { ig += tg; ie += te; }
-        }
-        unsigned rg = bg + ig - mg, re = be + ie - me;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const bool gt = (gm >> e) & 1u, eq = (em >> e) & 1u;
-          if (gt || (eq && re < quota)) {
-            const int pos = (int)(rg + min(re, quota));
-            if (pos >= R0 && pos < R1) {
-              if (pos - R0 < kMySelCap) sm.mysel[pos - R0] = base + e;
-              if (p.sel_out) p.sel_out[pos] = base + e;
-            }
+      for (int e = 0; e < 8; ++e) {
+        const bool gt = (gm >> e) & 1u, eq = (em >> e) & 1u;
+        if (gt || (eq && re < quota)) {
+          const int pos = (int)(rg + min(re, quota));
+          if (pos >= R0 && pos < R1) {
+            if (pos - R0 < kMySelCap) sm.mysel[pos - R0] = base + e;
+            if (p.sel_out) p.sel_out[pos] = base + e;
           }
-          rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
         }
+        rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
       }
     }
     fence_proxy_async();                      // the big buffer becomes a bulk-copy target next

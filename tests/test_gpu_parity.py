@@ -216,6 +216,48 @@ def test_forward_batched_per_token_masks(pb, toy, B):
     _forward_check(pb, p, 3, k1, k2, B=B)
 
 
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0)])
+def test_union_and_per_token_batch_paths_agree(pb, toy, bits, group):
+    """B > 1: one read of the weights for the union of the tokens' masks must give every
+    token the result of the per-token path (and of the oracle)."""
+    wl, p = toy
+    p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    B, t0 = 8, 8
+    res = []
+    for union in (1, 0):
+        pb.prox_ffn_set_union(p.h, union)
+        y = p.y_empty(B)
+        m = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        pb.prox_ffn_forward(p.h, p.t_x[t0:t0 + B], B, k1, k2, y)
+        pb.prox_ffn_last_mask(p.h, B, k2, m)
+        torch.cuda.synchronize()
+        res.append((y.cpu().numpy(), m.cpu().numpy().astype(np.int64)))
+    pb.prox_ffn_set_union(p.h, 1)
+    for b in range(B):
+        idx, score, sel_ref, thr = p.oracle_stage1(t0 + b, k1, k2)
+        for yv, mv in res:
+            check_mask(mv[b], score, sel_ref, thr, k2, p.F)
+            y_ref, _ = po.stage2(p.x[t0 + b], mv[b], p.wg, p.wu, p.wd)
+            assert check_y(yv[b], y_ref) < 1e-4
+    # stage-wise entry points on the union path, odd batch size
+    B = 3
+    sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+    sc = torch.empty(B, p.F, dtype=torch.float32, device="cuda")
+    y = p.y_empty(B)
+    pb.prox_stage1_mask(p.h, p.t_x[1:1 + B], B, k1, k2, sel, sc)
+    pb.prox_stage2_ffn(p.h, p.t_x[1:1 + B], B, sel, k2, y)
+    torch.cuda.synchronize()
+    for b in range(B):
+        idx, score, sel_ref, thr = p.oracle_stage1(1 + b, k1, k2)
+        mv = sel.cpu().numpy()[b].astype(np.int64)
+        check_mask(mv, score, sel_ref, thr, k2, p.F)
+        assert float(np.max(np.abs(sc.cpu().numpy()[b] - score)) / thr) < 2e-4
+        y_ref, _ = po.stage2(p.x[1 + b], mv, p.wg, p.wu, p.wd)
+        assert check_y(y.cpu().numpy()[b], y_ref) < 1e-4
+    assert pb.prox_last_device_status(p.h) == 0
+
+
 def test_forward_host_buffers(pb, toy):
     wl, p = toy
     p.quantize(4, 0)
