@@ -238,14 +238,14 @@ bool batch_path_ok(const prox_ffn* h, int B) {
   if (B < 2 || !h->u_in) return false;
   const size_t xs_bytes = (size_t)B * h->cfg.d_model * 2;
   const size_t red_bytes = (size_t)4 * kBT * 128 * (h->bits == 4 ? 8 : 4) * sizeof(float);
-  const size_t ubits = (size_t)B * ((h->cfg.d_ff + 31) / 32) * 4;
+  const size_t ubits = (size_t)(B + 2) * ((h->cfg.d_ff + 31) / 32) * 4;
   const size_t lim = (size_t)h->smem_optin - 4096;
   return xs_bytes <= lim && red_bytes <= lim && ubits <= lim;
 }
 
 prox_status_t launch_union(prox_ffn* h, const int* lists, int stride, const int* cnt, int k, int B, int n,
                            const void* x, int* ulist, int* nu, float* val, cudaStream_t st) {
-  const size_t smem = (size_t)B * ((n + 31) / 32) * sizeof(unsigned);
+  const size_t smem = (size_t)(B + 2) * ((n + 31) / 32) * sizeof(unsigned);
   static bool attr = false;
   if (!attr) { CK(cudaFuncSetAttribute(union_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
   {

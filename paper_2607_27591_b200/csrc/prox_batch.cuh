@@ -21,7 +21,7 @@ __global__ void __launch_bounds__(1024)
 union_kernel(const int* __restrict__ lists, int stride, const int* __restrict__ cnt, int k_static, int B,
              int n, const uint16_t* __restrict__ x, int* __restrict__ ulist, int* __restrict__ nu_out,
              float* __restrict__ val, int* __restrict__ status) {
-  extern __shared__ unsigned ubits[];                  // [B][nw]
+  extern __shared__ unsigned ubits[];                  // [B][nw] token bit sets, [nw] union, [nw] offsets
   __shared__ unsigned long long ws[33];
   const int nw = (n + 31) / 32;
   const int t = threadIdx.x;
@@ -36,34 +36,38 @@ union_kernel(const int* __restrict__ lists, int stride, const int* __restrict__ 
     }
   }
   __syncthreads();
+  // union words, their popcounts, and an exclusive scan of those (nw <= 2048)
+  unsigned* uw = ubits + (size_t)B * nw;               // [nw] union words, then [nw] word offsets
+  unsigned* woff = uw + nw;
   const int per = (nw + 1023) / 1024;                  // consecutive words per thread
   const int w0 = t * per;
   unsigned c = 0;
   for (int w = w0; w < w0 + per && w < nw; ++w) {
     unsigned u = 0;
     for (int b = 0; b < B; ++b) u |= ubits[b * nw + w];
+    uw[w] = u;
     c += __popc(u);
   }
   unsigned long long tot;
   unsigned off = (unsigned)block_scan_excl<1024>((unsigned long long)c, ws, &tot);
-  for (int w = w0; w < w0 + per && w < nw; ++w) {
-    unsigned u = 0;
-    for (int b = 0; b < B; ++b) u |= ubits[b * nw + w];
-    while (u) {
-      const int bit = __ffs(u) - 1;
-      u &= u - 1;
-      const int id = w * 32 + bit;
-      ulist[off] = id;
+  for (int w = w0; w < w0 + per && w < nw; ++w) { woff[w] = off; off += __popc(uw[w]); }
+  __syncthreads();
+  // one thread per index: members of the union write their row
+  for (int id = t; id < n; id += 1024) {
+    const int w = id >> 5, bit = id & 31;
+    const unsigned u = uw[w];
+    if ((u >> bit) & 1u) {
+      const unsigned pos = woff[w] + __popc(u & ((1u << bit) - 1u));
+      ulist[pos] = id;
       float v[kBT];
 #pragma unroll
       for (int b = 0; b < kBT; ++b) {
         const bool in = b < B && ((ubits[b * nw + w] >> bit) & 1u);
         v[b] = !in ? 0.f : (x ? __uint_as_float(((uint32_t)x[(size_t)b * n + id]) << 16) : 1.f);
       }
-      float4* dst = reinterpret_cast<float4*>(val + (size_t)off * kBT);
+      float4* dst = reinterpret_cast<float4*>(val + (size_t)pos * kBT);
       dst[0] = make_float4(v[0], v[1], v[2], v[3]);
       dst[1] = make_float4(v[4], v[5], v[6], v[7]);
-      ++off;
     }
   }
   if (t == 0) *nu_out = (int)tot;
@@ -109,24 +113,22 @@ proxy_batch_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
   const uint8_t* src = P + (size_t)strip * 512 + (size_t)word * 4;
   const __half* sbase = S + ((size_t)chunk * 2 + (wsel >> 1)) * CH + (wsel & 1) * CW;
   constexpr int U = 4;
+  int curg = -1;
+  float scl[CW];
+#pragma unroll
+  for (int c = 0; c < CW; ++c) scl[c] = 0.f;
   for (int r = w0; r < w1; r += U) {
     int ii[U];
     uint32_t wv[U];
     float4 xa[U], xb[U];
-    uint4 sv[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) ii[u] = (r + u < w1) ? __ldg(ulist + r + u) : -1;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      wv[u] = 0; sv[u] = make_uint4(0, 0, 0, 0);
+      wv[u] = 0;
       xa[u] = xb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (ii[u] >= 0) {
-        if (valid) {
-          wv[u] = __ldg(reinterpret_cast<const uint32_t*>(src + (size_t)ii[u] * row_bytes));
-          const __half* sp = sbase + (size_t)(ii[u] >> gshift) * nchunks * 2 * CH;
-          if (CW == 8) sv[u] = __ldg(reinterpret_cast<const uint4*>(sp));
-          else { const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(sp)); sv[u].x = t2.x; sv[u].y = t2.y; }
-        }
+        if (valid) wv[u] = __ldg(reinterpret_cast<const uint32_t*>(src + (size_t)ii[u] * row_bytes));
         xa[u] = __ldg(reinterpret_cast<const float4*>(xu + (size_t)(r + u) * kBT));
         xb[u] = __ldg(reinterpret_cast<const float4*>(xu + (size_t)(r + u) * kBT) + 1);
       }
@@ -134,8 +136,21 @@ proxy_batch_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (ii[u] < 0 || !valid) continue;
+      const int g = ii[u] >> gshift;
+      if (g != curg) {                                 // union rows ascend: a group's scales are loaded once
+        curg = g;
+        const __half* sp = sbase + (size_t)g * nchunks * 2 * CH;
+        uint4 sv = make_uint4(0, 0, 0, 0);
+        if (CW == 8) sv = __ldg(reinterpret_cast<const uint4*>(sp));
+        else { const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(sp)); sv.x = t2.x; sv.y = t2.y; }
+        const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          const __half2 h2 = *reinterpret_cast<const __half2*>(&sw[c >> 1]);
+          scl[c] = (c & 1) ? __high2float(h2) : __low2float(h2);
+        }
+      }
       float q[CW];
-      const uint32_t sw[4] = {sv[u].x, sv[u].y, sv[u].z, sv[u].w};
 #pragma unroll
       for (int c = 0; c < CW; ++c) {
         float code;
@@ -147,8 +162,7 @@ proxy_batch_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
         } else {
           code = __uint_as_float(__byte_perm(wv[u], 0x4B000000u, 0x7650u | c)) - 8388736.0f;
         }
-        const __half2 h2 = *reinterpret_cast<const __half2*>(&sw[c >> 1]);
-        q[c] = code * ((c & 1) ? __high2float(h2) : __low2float(h2));
+        q[c] = code * scl[c];
       }
       const float xt[kBT] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
 #pragma unroll
