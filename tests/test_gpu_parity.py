@@ -339,6 +339,25 @@ def test_fused_all_zero_input(pb, toy):
     assert float(y.abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("D,F,k1,k2,bits,group", [
+    (16384, 1024, 4915, 239, 4, 128),      # widest d_model the library takes (fused kernel not used: step-wise path)
+    (128, 65536, 38, 15270, 4, 0),         # narrowest d_model, widest d_ff
+    (8192, 320, 2458, 75, 8, 128),         # ragged last strip, 8-bit codes, two down-projection groups
+    (384, 448, 115, 104, 4, 128),          # sizes that are no multiple of the strip or chunk steps
+])
+def test_extreme_shapes(pb, D, F, k1, k2, bits, group):
+    wg, wu, wd, x = inputs.make_small(D, F, 3, seed=D + F)
+    p = Problem(pb, wg, wu, wd, x, max_batch=2)
+    try:
+        p.quantize(bits, group)
+        for t in range(2):
+            _forward_check(pb, p, t, k1, k2)
+        _forward_check(pb, p, 1, k1, k2, B=2)
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
+
+
 # --------------------------------------------------------- threshold variant
 def test_threshold_variant(pb, toy):
     wl, p = toy
