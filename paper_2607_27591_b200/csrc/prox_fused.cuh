@@ -405,13 +405,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     const uint32_t wbuf = wscale + (uint32_t)(kScaleGroupsPerWarp * SCB);
     for (int item = cta; item < nitems; item += G) {
       const int strip = item % p.nstrips, ks = item / p.nstrips;
-      const int r0 = (int)(((long long)k1 * ks) / p.ksplit), r1 = (int)(((long long)k1 * (ks + 1)) / p.ksplit);
+      // 32-bit arithmetic on purpose (k1 <= 16384, ks < 64): a 64-bit division costs about a microsecond here
+      const int r0 = (int)(((unsigned)k1 * (unsigned)ks) / (unsigned)p.ksplit);
+      const int r1 = (int)(((unsigned)k1 * (unsigned)(ks + 1)) / (unsigned)p.ksplit);
       float tot[NACC];
 #pragma unroll
       for (int c = 0; c < NACC; ++c) tot[c] = 0.f;
       if (warp < kFusedConsumerWarps) {
-        const int w0 = r0 + (int)(((long long)(r1 - r0) * warp) / kFusedConsumerWarps);
-        const int w1 = r0 + (int)(((long long)(r1 - r0) * (warp + 1)) / kFusedConsumerWarps);
+        const int w0 = r0 + (int)(((unsigned)(r1 - r0) * (unsigned)warp) / (unsigned)kFusedConsumerWarps);
+        const int w1 = r0 + (int)(((unsigned)(r1 - r0) * (unsigned)(warp + 1)) / (unsigned)kFusedConsumerWarps);
         const int nrows = w1 - w0;
         const int seg = (int)min((size_t)512, row_bytes - (size_t)strip * 512);
         const bool lane_valid = lane * 16 < seg;
@@ -581,7 +583,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   if (tid == 0) {
     __threadfence();                          // cumulative: publishes the block's writes seen through the barrier above
     const unsigned long long old = atomicAdd(p.bar_count, 1ull);
-    const unsigned long long target = (old / (unsigned long long)G + 1ull) * (unsigned long long)G;
+    // the count is reset by the host long before 2^32 calls; the low word is enough for the division
+    const unsigned long long target = old - (unsigned long long)((unsigned)old % (unsigned)G) + (unsigned long long)G;
     bool ok = (old + 1ull == target);
     for (unsigned it = 0; !ok && it < kSpinLimit; ++it) {
       unsigned long long cur;
@@ -597,7 +600,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   PROX_TRACE(4);
 
   // ---------------------------------------- C: channel mask (top-k2 of the scores)
-  const int R0 = (int)(((long long)k2 * cta) / G), R1 = (int)(((long long)k2 * (cta + 1)) / G);
+  // k2 <= 65536 and cta < 65536 would overflow 32 bits only beyond any real grid (k2 * G < 2^31 is checked on the host)
+  const int R0 = (int)(((unsigned)k2 * (unsigned)cta) / (unsigned)G), R1 = (int)(((unsigned)k2 * (unsigned)(cta + 1)) / (unsigned)G);
   if (alive) {
     unsigned* skey = reinterpret_cast<unsigned*>(big);
     const bool in_smem = (size_t)F * 4 + (size_t)kCandCap * 8 <= (size_t)p.big_bytes;
