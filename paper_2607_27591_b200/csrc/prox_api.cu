@@ -51,6 +51,7 @@ struct prox_ffn {
                             // (64-bit, [2048..2049]), [2050] finish ticket
   int smem_optin;           // largest dynamic shared memory a block may ask for
   int coop;                 // device supports cooperative launch
+  int sel_unordered;        // the last forward left its mask in the persistent kernel's own order
   int use_fused;            // batch-1 forward runs as one persistent kernel
   int use_union;            // batch > 1 reads weights once for the union of the tokens' masks
   unsigned long long* trace;  // optional phase time stamps of the persistent kernel (debug)
@@ -350,7 +351,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   if (pl.big_bytes < kFusedConsumerWarps * (kScaleGroupsPerWarp * scb + kProxyRowsInFlight * 512)) return pl;   // proxy row buffers
   if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;      // reduction scratch
   if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
-  if ((k2 + G - 1) / G > kMySelCap) return pl;
+  if ((k2 + G - 1) / G + 2 > kMySelCap) return pl;       // a block's share: definite part + part of the threshold bin
   pl.nstrips = nstrips_for(F, h->bits);
   // row split: fill the grid evenly (items = strips * ksplit run in rounds of G blocks)
   int best = 1;
@@ -599,8 +600,9 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   if (B == 1) {
     const FusedPlan pl = plan_fused(h, k1, k2);
-    if (pl.ok) return launch_fused(h, pl, x, k1, k2, y, h->sel, st);
+    if (pl.ok) { h->sel_unordered = 1; return launch_fused(h, pl, x, k1, k2, y, h->sel, st); }
   }
+  h->sel_unordered = 0;
   if (h->use_union && batch_path_ok(h, B)) {
     if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st)) != PROX_OK) return s;
     return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st);
@@ -661,9 +663,16 @@ prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on) {
 
 prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev, void* stream) {
   if (!h || !sel_dev || B < 1 || B > h->cfg.max_batch || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (B == 1 && h->sel_unordered) {
+    // the persistent kernel lists the kept channels in its own order; the score buffer is free between calls
+    LaunchScope ls(h, kKChannel, st);
+    mask_ascending_kernel<<<1, 1024, 0, st>>>(h->sel, k2, h->cfg.d_ff, reinterpret_cast<int*>(h->scores), sel_dev);
+    CK(cudaGetLastError());
+    return PROX_OK;
+  }
   CK(cudaMemcpy2DAsync(sel_dev, (size_t)k2 * sizeof(int), h->sel, (size_t)h->cfg.d_ff * sizeof(int),
-                       (size_t)k2 * sizeof(int), (size_t)B, cudaMemcpyDeviceToDevice,
-                       static_cast<cudaStream_t>(stream)));
+                       (size_t)k2 * sizeof(int), (size_t)B, cudaMemcpyDeviceToDevice, st));
   return PROX_OK;
 }
 

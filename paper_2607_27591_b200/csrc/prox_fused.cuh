@@ -26,6 +26,8 @@ namespace prox {
 
 constexpr int kFusedConsumerWarps = 16;
 constexpr int kFusedConsumers = kFusedConsumerWarps * 32;       // 512
+constexpr int kSettlerWarps = 8;                                 // consumer warps that finish the channel mask
+constexpr int kSettlers = kSettlerWarps * 32;
 constexpr int kFusedProducers = 4;                               // warps whose lane 0 issues bulk copies
 constexpr int kFusedThreads = kFusedConsumers + 32 * kFusedProducers;   // 640
 constexpr int kFusedWarps = kFusedThreads / 32;                 // 20
@@ -111,6 +113,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 #define PROX_TRACE(k) do { if (p.trace && tid == 0) p.trace[(size_t)cta * 32 + (k)] = global_ns(); } while (0)
+__device__ __forceinline__ void settler_sync() {      // the lower half of the consumer warps
+  asm volatile("bar.sync 3, %0;" ::"n"(kSettlers) : "memory");
+}
 __device__ __forceinline__ void consumer_sync() {     // the 512 consumer threads only
   asm volatile("bar.sync 1, %0;" ::"n"(kFusedConsumers) : "memory");
 }
@@ -149,87 +154,71 @@ __device__ __forceinline__ bool slot_wait(uint32_t bar, volatile unsigned* seen,
   return true;
 }
 
-// Exclusive prefix over the lanes of a warp of popc(m8), m8 an 8-bit mask per
-// lane: eight ballots instead of a five-step shuffle scan (shuffles are slow here).
-__device__ __forceinline__ unsigned lane_prefix8(unsigned m8, unsigned lt_mask) {
-  unsigned pre = 0;
-#pragma unroll
-  for (int e = 0; e < 8; ++e) pre += __popc(__ballot_sync(0xffffffffu, (m8 >> e) & 1u) & lt_mask);
-  return pre;
+// The selection phases run once per call on every block, over code that is cold
+// in the instruction caches: their time is set by the number of instructions
+// fetched, not executed.  They are therefore written as small loops (one key per
+// lane and trip) and the helpers below are shared between the phases.
+
+__device__ __forceinline__ unsigned warp_scan_incl(unsigned v, int lane) {
+#pragma unroll 1
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
 }
 
-// k-th largest bin of hist[0..NBINS) counted from the top, with two block
-// barriers: warps scan their bins with shuffles, every thread then adds up the
-// totals of the warps in front of it.  Result in res[0] (bin), res[1] (above).
-template <int NT, int NBINS>
-__device__ __forceinline__ void find_kth_fast(const unsigned* hist, unsigned k, unsigned* wsum, unsigned* res) {
-  constexpr int PER = (NBINS + NT - 1) / NT;
-  constexpr int NW = NT / 32;
-  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  unsigned loc[PER];
-  unsigned sum = 0;
-#pragma unroll
-  for (int q = 0; q < PER; ++q) {
-    const int bin = NBINS - 1 - (t * PER + q);
-    loc[q] = (bin >= 0) ? hist[bin] : 0u;
-    sum += loc[q];
+// k-th largest (k >= 1, counted from the top) among the 32 * BPL bins that end
+// below index `top`.  One warp; every lane returns the same bin and the count
+// above it.  Lane l owns the l-th slice of BPL bins from the top.
+template <int BPL>
+__device__ __forceinline__ unsigned kth_in_segment(const unsigned* hist, int top, unsigned k, int lane, unsigned* above) {
+  const int base = top - (lane + 1) * BPL;
+  unsigned s = 0;
+#pragma unroll 1
+  for (int j = 0; j < BPL; ++j) s += hist[base + j];
+  const unsigned inc = warp_scan_incl(s, lane);
+  const unsigned ex = inc - s;
+  const unsigned m = __ballot_sync(0xffffffffu, ex < k && k <= inc);
+  const int src = m ? (__ffs(m) - 1) : 31;
+  unsigned run = __shfl_sync(0xffffffffu, ex, src);
+  const int b0 = top - (src + 1) * BPL;                 // all lanes walk the same slice (broadcast reads)
+  unsigned bin = (unsigned)b0, ab = run;
+#pragma unroll 1
+  for (int j = BPL - 1; j >= 0; --j) {
+    const unsigned c = hist[b0 + j];
+    if (run < k && k <= run + c) { bin = (unsigned)(b0 + j); ab = run; }
+    run += c;
   }
-  unsigned inc = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned v = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += v;
-  }
-  if (lane == 31) wsum[warp] = inc;
-  __syncthreads();
-  unsigned pre = 0;
-#pragma unroll
-  for (int w = 0; w < NW; ++w) { const unsigned v = wsum[w]; pre += (w < warp) ? v : 0u; }
-  const unsigned ex = pre + inc - sum;
-  if (ex < k && k <= ex + sum) {
-    unsigned run = ex;
-#pragma unroll
-    for (int q = 0; q < PER; ++q) {
-      if (run < k && k <= run + loc[q]) { res[0] = (unsigned)(NBINS - 1 - (t * PER + q)); res[1] = run; }
-      run += loc[q];
-    }
-  }
-  __syncthreads();
-}
-
-// Same for NBINS <= 256, done by one warp alone (every warp may call it with the
-// same arguments and gets the same answer; no block barrier).  Returns the bin
-// and writes the count above it.
-template <int NBINS>
-__device__ __forceinline__ unsigned find_kth_warp(const unsigned* hist, unsigned k, unsigned* above) {
-  constexpr int PER = NBINS / 32;
-  const int lane = threadIdx.x & 31;
-  unsigned loc[PER];
-  unsigned sum = 0;
-#pragma unroll
-  for (int q = 0; q < PER; ++q) { loc[q] = hist[NBINS - 1 - (lane * PER + q)]; sum += loc[q]; }
-  unsigned inc = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned v = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += v;
-  }
-  const unsigned ex = inc - sum;
-  const bool mine = ex < k && k <= ex + sum;
-  unsigned bin = 0, ab = 0;
-  if (mine) {
-    unsigned run = ex;
-#pragma unroll
-    for (int q = 0; q < PER; ++q) {
-      if (run < k && k <= run + loc[q]) { bin = (unsigned)(NBINS - 1 - (lane * PER + q)); ab = run; }
-      run += loc[q];
-    }
-  }
-  const unsigned who = __ballot_sync(0xffffffffu, mine);
-  const int src = who ? (__ffs(who) - 1) : 0;
-  bin = __shfl_sync(0xffffffffu, bin, src);
-  ab = __shfl_sync(0xffffffffu, ab, src);
   *above = ab;
+  return bin;
+}
+
+// Same over 512 * BPL bins with the whole block (one block barrier inside):
+// warps 0..15 total their segment, then every warp locates the segment and
+// finishes on its own, so the result is in the registers of every thread.
+template <int BPL>
+__device__ __forceinline__ unsigned kth_in_block(const unsigned* hist, unsigned k, unsigned* wsum, int lane, int warp,
+                                                 unsigned* above) {
+  constexpr int NB = 512 * BPL, SEG = 32 * BPL;
+  if (warp < 16) {
+    const int base = NB - warp * SEG - (lane + 1) * BPL;
+    unsigned s = 0;
+#pragma unroll 1
+    for (int j = 0; j < BPL; ++j) s += hist[base + j];
+    s = __reduce_add_sync(0xffffffffu, s);
+    if (lane == 0) wsum[warp] = s;
+  }
+  __syncthreads();
+  const unsigned v = (lane < 16) ? wsum[lane] : 0u;
+  const unsigned inc = warp_scan_incl(v, lane);
+  const unsigned ex = inc - v;
+  const unsigned m = __ballot_sync(0xffffffffu, ex < k && k <= inc);
+  const int seg = m ? (__ffs(m) - 1) : 15;
+  const unsigned aseg = __shfl_sync(0xffffffffu, ex, seg);
+  unsigned ab;
+  const unsigned bin = kth_in_segment<BPL>(hist, NB - seg * SEG, k - aseg, lane, &ab);
+  *above = aseg + ab;
   return bin;
 }
 
@@ -251,6 +240,12 @@ struct FusedSmem {
   unsigned ncand;
   unsigned ncand2;
   unsigned prod_seq;       // rows the producers have armed so far (for the give-up path)
+  unsigned next_c;         // next channel of the batch to take in the gate/up phase
+  int nready;              // entries of mysel that are final (the definite share first, all of them later)
+  int keys_done;           // the consumer warps no longer read the keys near the end of the big buffer
+  int c_done;              // ... nor the list of the threshold bin's members
+  int keys_s0, keys_s1;    // ring slots [s0, s1) that overlap the keys
+  int list_s0, list_s1;    // ... and the list
   unsigned slot_use[kMaxSlots];   // uses of each ring slot whose data has been seen complete
 };
 
@@ -279,7 +274,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     mbar_init(smem_u32(&sm.mbar_empty[tid]), kEmptyCount);
     fence_mbar_init();
   }
-  if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; }
+  if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; }
   if (tid < kMaxSlots) sm.slot_use[tid] = 0;
   {
     const uint4* xg = reinterpret_cast<const uint4*>(p.x);
@@ -296,95 +291,70 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   PROX_TRACE(1);
 
   // ------------------------------------------------- A: input mask (top-k1 of |x|)
-  // A warp takes 256 consecutive inputs at a time, 8 per lane (one 16-byte load).
   {
-    const int nvec = D / 8;                               // 8-key vectors
-    const int nchk = (nvec + 31) / 32;                    // 256-key chunks (<= 64)
+    const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
+    const bool all = k1 >= D;
     unsigned T = 0, quota = 0;
-    if (k1 < D) {
-      // level 1: 10 bits (exponent and two mantissa bits), level 2: the other 5
-      for (int q = warp; q < nchk; q += kFusedWarps) {
-        const int v = q * 32 + lane;
-        if (v < nvec) {
-          const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
-          const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            atomicAdd(&sm.hist[(w[e] & 0x7fffu) >> 5], 1u);
-            atomicAdd(&sm.hist[(w[e] >> 21) & 0x3ffu], 1u);
-          }
-        }
+    if (!all) {
+      // level 1: the top 10 of the 15 key bits; level 2: the other 5
+#pragma unroll 1
+      for (int i = tid; i < D / 2; i += NT) {
+        const uint32_t w = xs32[i];
+        atomicAdd(&sm.hist[(w >> 5) & 0x3ffu], 1u);
+        atomicAdd(&sm.hist[(w >> 21) & 0x3ffu], 1u);
       }
       __syncthreads();
       PROX_TRACE(10);
-      find_kth_fast<NT, 1024>(sm.hist, (unsigned)k1, sm.wsum, sm.res);
-      const unsigned bin1 = sm.res[0], above1 = sm.res[1];
+      unsigned above1;
+      const unsigned bin1 = kth_in_block<2>(sm.hist, (unsigned)k1, sm.wsum, lane, warp, &above1);
       PROX_TRACE(11);
-      for (int q = warp; q < nchk; q += kFusedWarps) {
-        const int v = q * 32 + lane;
-        if (v < nvec) {
-          const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
-          const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const unsigned k0 = w[e] & 0x7fffu, k1b = (w[e] >> 16) & 0x7fffu;
-            if ((k0 >> 5) == bin1) atomicAdd(&sm.hist2[k0 & 31u], 1u);
-            if ((k1b >> 5) == bin1) atomicAdd(&sm.hist2[k1b & 31u], 1u);
-          }
-        }
+#pragma unroll 1
+      for (int i = tid; i < D / 2; i += NT) {
+        const uint32_t w = xs32[i];
+        const unsigned ka = w & 0x7fffu, kb = (w >> 16) & 0x7fffu;
+        if ((ka >> 5) == bin1) atomicAdd(&sm.hist2[ka & 31u], 1u);
+        if ((kb >> 5) == bin1) atomicAdd(&sm.hist2[kb & 31u], 1u);
       }
       __syncthreads();
       PROX_TRACE(12);
       unsigned above2;
-      const unsigned bin2 = find_kth_warp<32>(sm.hist2, (unsigned)k1 - above1, &above2);
+      const unsigned bin2 = kth_in_segment<1>(sm.hist2, 32, (unsigned)k1 - above1, lane, &above2);
       T = (bin1 << 5) | bin2;
       quota = (unsigned)k1 - above1 - above2;      // ties at T to accept, lowest index first
       PROX_TRACE(13);
     }
-    // Ordered compaction.  A warp keeps the kept/tie masks of its chunks in
-    // registers, counts them with one warp reduction and prefixes them with ballots.
-    unsigned* ccnt = sm.hist;                              // reuse: [1024 + q] packed counts of chunk q
-    constexpr int MAXC = 4;                                // chunks per warp (64 chunks / 20 warps)
-    unsigned gmv[MAXC], emv[MAXC], pgv[MAXC], pev[MAXC];
+    // Ordered compaction: a consumer thread owns a run of 8-input groups, counts its kept
+    // inputs and its ties (packed in one word), and places them behind those of the threads
+    // in front (one warp scan plus the totals of the warps in front).
+    const int ngrp = D / 8, gpt = (ngrp + kFusedConsumers - 1) / kFusedConsumers;
+    const int g0 = min(ngrp, tid * gpt), g1 = (tid < kFusedConsumers) ? min(ngrp, g0 + gpt) : g0;
+    unsigned cnt = 0;
+#pragma unroll 1
+    for (int g = g0; g < g1; ++g) {
+      const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
+      const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
-    for (int sidx = 0; sidx < MAXC; ++sidx) {
-      const int q = warp + sidx * kFusedWarps;
-      gmv[sidx] = emv[sidx] = pgv[sidx] = pev[sidx] = 0;
-      if (q < nchk) {                                      // warp-uniform
-        const int v = q * 32 + lane;
-        unsigned gm = 0, em = 0;
-        if (v < nvec) {
-          const uint4 kv = reinterpret_cast<const uint4*>(xs)[v];
-          const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const unsigned key = (w[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
-            gm |= ((k1 >= D || key > T) ? 1u : 0u) << e;
-            em |= ((k1 < D && key == T) ? 1u : 0u) << e;
-          }
-        }
-        gmv[sidx] = gm; emv[sidx] = em;
-        pgv[sidx] = lane_prefix8(gm, lt_mask);
-        pev[sidx] = lane_prefix8(em, lt_mask);
-        const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(gm) | ((unsigned)__popc(em) << 16));
-        if (lane == 0) ccnt[1024 + q] = tot;
+      for (int e = 0; e < 8; ++e) {
+        const unsigned key = (w4[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
+        cnt += ((all || key > T) ? 1u : 0u) | ((!all && key == T) ? 0x10000u : 0u);
       }
     }
+    const unsigned inc = warp_scan_incl(cnt, lane);
+    if (lane == 31) sm.wsum[warp] = inc;
     __syncthreads();
     PROX_TRACE(14);
-#pragma unroll
-    for (int sidx = 0; sidx < MAXC; ++sidx) {
-      const int q = warp + sidx * kFusedWarps;
-      if (q < nchk) {
-        unsigned bsum = 0;                                 // counts of the chunks in front (<= 64)
-        for (int j = lane; j < q; j += 32) bsum += ccnt[1024 + j];
-        bsum = __reduce_add_sync(0xffffffffu, bsum);
-        unsigned rg = (bsum & 0xffffu) + pgv[sidx], re = (bsum >> 16) + pev[sidx];
-        const int v = q * 32 + lane;
+    {
+      const unsigned ex = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u) + inc - cnt;
+      unsigned rg = ex & 0xffffu, re = ex >> 16;
+#pragma unroll 1
+      for (int g = g0; g < g1; ++g) {
+        const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
+        const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const bool gt = (gmv[sidx] >> e) & 1u, eq = (emv[sidx] >> e) & 1u;
-          if (gt || (eq && re < quota)) idx16[rg + min(re, quota)] = (uint16_t)(v * 8 + e);
+          const unsigned key = (w4[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
+          const bool gt = all || key > T, eq = !all && key == T;
+          if (gt || (eq && re < quota)) idx16[rg + min(re, quota)] = (uint16_t)(g * 8 + e);
           rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
         }
       }
@@ -600,204 +570,316 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   PROX_TRACE(4);
 
   // ---------------------------------------- C: channel mask (top-k2 of the scores)
-  // k2 <= 65536 and cta < 65536 would overflow 32 bits only beyond any real grid (k2 * G < 2^31 is checked on the host)
-  const int R0 = (int)(((unsigned)k2 * (unsigned)cta) / (unsigned)G), R1 = (int)(((unsigned)k2 * (unsigned)(cta + 1)) / (unsigned)G);
+  // The first histogram level tells which channels are kept whatever the exact
+  // threshold turns out to be (their bin lies above the threshold bin b1:
+  // "definite", nd of them) and which are still open (the nb1 members of b1).
+  // The kept list is laid out as [definite, ascending][kept members of b1,
+  // ascending]; block c owns the c-th share of either part.  Its definite share
+  // is known after two passes over the scores, so its weight rows start to stream
+  // while the consumer warps still settle the threshold inside b1.
+  int n_mine = 0;
   if (alive) {
-    unsigned* skey = reinterpret_cast<unsigned*>(big);
-    const bool in_smem = (size_t)F * 4 + (size_t)kCandCap * 8 <= (size_t)p.big_bytes;
-    unsigned* cand_key = reinterpret_cast<unsigned*>(big + (in_smem ? (size_t)F * 4 : 0));
-    int* cand_idx = reinterpret_cast<int*>(cand_key + kCandCap);
+    // Shared-memory plan: the keys (score bits) sit near the END of the big buffer and the
+    // ascending list of b1's members behind them (before them if it is long): the ring fills
+    // from slot 0 and reaches those slots last.
+    constexpr uint32_t kListFixed = 8192;                  // room for 1024 members behind the keys
+    const bool in_smem = (size_t)F * 4 + kListFixed + 256 <= (size_t)p.big_bytes;
+    const uint32_t list_fixed_off = ((uint32_t)p.big_bytes - kListFixed) & ~127u;
+    const uint32_t key_off = in_smem ? ((list_fixed_off - (uint32_t)F * 4u) & ~127u) : 0u;
+    const uint32_t skey_u32 = big_u32 + key_off;
     const unsigned* gkey = reinterpret_cast<const unsigned*>(p.scores);
-    {
-      unsigned hv[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { const int i = tid + q * NT; hv[q] = (i < 2048) ? __ldcg(p.ghist + i) : 0u; }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { const int i = tid + q * NT; if (i < 2048) sm.hist[i] = hv[q]; }
-      if (tid < 256) sm.hist2[tid] = 0;
+    auto key_at = [&](int i) -> unsigned {
+      unsigned v;
+      if (in_smem) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(skey_u32 + (uint32_t)i * 4u));
+      else v = __ldcg(gkey + i);
+      return v;
+    };
+    auto key4_at = [&](int i) -> uint4 {                  // i % 4 == 0
+      return in_smem ? lds128(skey_u32 + (uint32_t)i * 4u) : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
+    };
+    if (tid < 512) cp_async16(smem_u32(sm.hist) + (uint32_t)tid * 16u, p.ghist + tid * 4);
+    cp_async_commit();
+    if (in_smem) {
+#pragma unroll 1
+      for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
     }
+    cp_async_commit();
+    if (tid < 256) sm.hist2[tid] = 0;
+    cp_async_wait<1>();                                    // the histogram (the keys may still be on their way)
     __syncthreads();
     PROX_TRACE(16);
-    find_kth_fast<NT, 2048>(sm.hist, (unsigned)k2, sm.wsum, sm.res);
-    const unsigned b1 = sm.res[0];
-    unsigned kk = (unsigned)k2 - sm.res[1];
+    unsigned nd;                                           // channels above bin b1
+    const unsigned b1 = kth_in_block<4>(sm.hist, (unsigned)k2, sm.wsum, lane, warp, &nd);
+    const unsigned kk = (unsigned)k2 - nd;                 // members of b1 to keep (>= 1)
+    const unsigned nb1 = sm.hist[b1];
+    uint32_t list_off = list_fixed_off;
+    bool staged = in_smem;                                 // the same in every block
+    if (in_smem && nb1 * 8u > kListFixed) {
+      if ((size_t)nb1 * 8 + 128 <= (size_t)key_off) list_off = (key_off - nb1 * 8u) & ~127u;
+      else staged = false;
+    }
+    const int per = ((F + 32 * kFusedWarps - 1) / (32 * kFusedWarps)) * 32;        // channels per warp run (slow path)
+    const int i0 = min(F, warp * per), i1 = min(F, i0 + per);
+    cp_async_wait<0>();
     PROX_TRACE(17);
-    // scores -> shared memory, 256 channels per warp step (8 keys per lane);
-    // members of the threshold bin become candidates; channels above it are
-    // counted per chunk right away (they are selected whatever the exact threshold).
-    unsigned* ccnt = sm.hist;                              // [q] kept, [1024 + q] ties, per 256-channel chunk
-    const int nchk = (F + 255) / 256;                      // <= 256
-    __syncthreads();                                       // find_kth_fast is done with sm.hist
-    for (int q = warp; q < nchk; q += kFusedWarps) {
-      const int base = q * 256 + lane * 8;
-      uint4 kv[2];
+    __syncthreads();                                       // the keys are there for everyone; wsum is free again
+    if (staged) {
+      // k2 * G < 2^31 is checked on the host, so the share bounds fit 32 bits
+      const int Rd0 = (int)((nd * (unsigned)cta) / (unsigned)G), Rc0 = (int)((kk * (unsigned)cta) / (unsigned)G);
+      const int ndm = min((int)((nd * (unsigned)(cta + 1)) / (unsigned)G) - Rd0, kMySelCap);
+      const int ncm = min((int)((kk * (unsigned)(cta + 1)) / (unsigned)G) - Rc0, kMySelCap - ndm);
+      const int Rd1 = Rd0 + ndm, Rc1 = Rc0 + ncm;
+      n_mine = ndm + ncm;
+      // pass 1: a consumer thread owns a run of 4-channel groups and counts its definite
+      // channels and its members of b1 (packed in one word); one warp scan, warp totals
+      const int nq = F / 4, qpt = (nq + kFusedConsumers - 1) / kFusedConsumers;
+      const int q0 = min(nq, tid * qpt), q1 = (tid < kFusedConsumers) ? min(nq, q0 + qpt) : q0;
+      unsigned cnt = 0;
+#pragma unroll 1
+      for (int q = q0; q < q1; ++q) {
+        const uint4 kv = key4_at(q * 4);
+        const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh)
-        kv[hh] = (base + hh * 4 < F) ? __ldcg(reinterpret_cast<const uint4*>(gkey + base + hh * 4)) : make_uint4(0, 0, 0, 0);
-      unsigned hi = 0;
+        for (int e = 0; e < 4; ++e) {
+          const unsigned bin = k4[e] >> 20;
+          cnt += ((bin > b1) ? 1u : 0u) | ((bin == b1) ? 0x10000u : 0u);
+        }
+      }
+      const unsigned inc = warp_scan_incl(cnt, lane);
+      if (lane == 31) sm.wsum[warp] = inc;
+      if (tid == 0) {
+        const uint32_t rb = (uint32_t)D * 2u;
+        sm.keys_s0 = (int)(key_off / rb); sm.keys_s1 = (int)((key_off + (uint32_t)F * 4u + rb - 1u) / rb);
+        sm.list_s0 = (int)(list_off / rb); sm.list_s1 = (int)((list_off + nb1 * 8u + rb - 1u) / rb);
+        sm.nready = ndm; sm.keys_done = (ncm == 0) ? 1 : 0; sm.c_done = (ncm == 0) ? 1 : 0;
+      }
+      __syncthreads();
+      PROX_TRACE(18);
+      // pass 2: the threads whose definite channels meet the block's share write them out
+      const unsigned ex = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u) + inc - cnt;
+      {
+        int dpos = (int)(ex & 0xffffu);
+        const int cdef = (int)(cnt & 0xffffu);
+        if (cdef > 0 && dpos < Rd1 && dpos + cdef > Rd0) {
+#pragma unroll 1
+          for (int q = q0; q < q1; ++q) {
+            const uint4 kv = key4_at(q * 4);
+            const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int i = base + hh * 4;
-        if (i < F) {
-          if (in_smem) *reinterpret_cast<uint4*>(skey + i) = kv[hh];
-          const unsigned kk4[4] = {kv[hh].x, kv[hh].y, kv[hh].z, kv[hh].w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const unsigned bin = kk4[e] >> 20;
-            hi += (bin > b1) ? 1u : 0u;
-            if (bin == b1) {
-              const unsigned slot = atomicAdd(&sm.ncand, 1u);
-              if (slot < (unsigned)kCandCap) {
-                cand_key[slot] = kk4[e]; cand_idx[slot] = i + e;
-                atomicAdd(&sm.hist2[(kk4[e] >> 12) & 255u], 1u);
+            for (int e = 0; e < 4; ++e) {
+              if ((k4[e] >> 20) > b1) {
+                if (dpos >= Rd0 && dpos < Rd1) {
+                  sm.mysel[dpos - Rd0] = q * 4 + e;
+                  if (p.sel_out) p.sel_out[dpos] = q * 4 + e;
+                }
+                ++dpos;
               }
             }
           }
         }
       }
-      hi = __reduce_add_sync(0xffffffffu, hi);
-      if (lane == 0) { ccnt[q] = hi; ccnt[1024 + q] = 0; }
-    }
-    __syncthreads();
-    const unsigned ncand = sm.ncand;
-    PROX_TRACE(18);
-    unsigned T = 0, quota = 0;
-    bool have_T = false;
-    if (ncand <= (unsigned)kCandCap) {
-      // second level (bits 19..12) over the candidates, found by every warp on its own
-      unsigned above2;
-      const unsigned b2 = find_kth_warp<256>(sm.hist2, kk, &above2);
-      const unsigned kk2 = kk - above2;
-      const unsigned pre2 = (b1 << 8) | b2;
-      for (unsigned c = tid; c < ncand; c += NT) {
-        const unsigned key = cand_key[c];
-        if ((key >> 12) == pre2) {
-          const unsigned slot = atomicAdd(&sm.ncand2, 1u);
-          if (slot < (unsigned)kCand2Cap) { sm.cand2_key[slot] = key; sm.cand2_idx[slot] = cand_idx[c]; }
-        }
-      }
-      __syncthreads();
-      const unsigned n2 = sm.ncand2;
-      PROX_TRACE(19);
-      if (n2 <= (unsigned)kCand2Cap) {
-        // rank the few that are left by (score descending, channel ascending)
-        if (tid < (int)n2) {
-          const unsigned key = sm.cand2_key[tid];
-          const int id = sm.cand2_idx[tid];
-          unsigned rank = 0, same_before = 0;
-          for (unsigned c = 0; c < n2; ++c) {
-            const unsigned ok = sm.cand2_key[c];
-            const int oi = sm.cand2_idx[c];
-            rank += (ok > key || (ok == key && oi < id)) ? 1u : 0u;
-            same_before += (ok == key && oi < id) ? 1u : 0u;
+      fence_proxy_async();                      // the big buffer becomes a bulk-copy target next
+      __syncthreads();                          // the producer warps leave for the ring here
+      PROX_TRACE(21);
+      if (ncm > 0 && warp < kFusedConsumerWarps) {
+        // ---- consumer warps only (named barrier): list b1's members in channel order ...
+        const uint32_t lkey_u32 = big_u32 + list_off, lidx_u32 = lkey_u32 + nb1 * 4u;
+        auto lds32 = [](uint32_t a) -> unsigned { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v; };
+        auto sts32 = [](uint32_t a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); };
+        if (cnt >> 16) {
+          unsigned cpos = ex >> 16;
+#pragma unroll 1
+          for (int q = q0; q < q1; ++q) {
+            const uint4 kv = key4_at(q * 4);
+            const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if ((k4[e] >> 20) == b1) {
+                if (cpos < nb1) { sts32(lkey_u32 + cpos * 4u, k4[e]); sts32(lidx_u32 + cpos * 4u, (unsigned)(q * 4 + e)); }
+                ++cpos;
+              }
+            }
           }
-          if (rank == kk2 - 1u) { sm.res[2] = key; sm.res[3] = same_before + 1u; }
         }
-        __syncthreads();
-        T = sm.res[2]; quota = sm.res[3];
+        // The upper half of the consumer warps goes on to the gate/up rows that are streaming in
+        // already; the lower half ("settlers") finishes the mask and joins them later.
+        if (warp >= kSettlerWarps) {
+          asm volatile("bar.arrive 2, %0;" ::"n"(kFusedConsumers) : "memory");
+        } else {
+        asm volatile("bar.sync 2, %0;" ::"n"(kFusedConsumers) : "memory");      // the list is complete, the keys are free
+        if (tid == 0) *reinterpret_cast<volatile int*>(&sm.keys_done) = 1;
+        PROX_TRACE(15);
+        // ... settle the threshold inside b1: histogram of bits 19..12, then the few left ...
+#pragma unroll 1
+        for (unsigned c = tid; c < nb1; c += kSettlers)
+          atomicAdd(&sm.hist2[(lds32(lkey_u32 + c * 4u) >> 12) & 255u], 1u);
+        settler_sync();
+        unsigned above2;
+        const unsigned b2 = kth_in_segment<8>(sm.hist2, 256, kk, lane, &above2);     // every warp on its own
+        unsigned kk2 = kk - above2;
+        const unsigned pre2 = (b1 << 8) | b2;
+#pragma unroll 1
+        for (unsigned c = tid; c < nb1; c += kSettlers) {
+          const unsigned key = lds32(lkey_u32 + c * 4u);
+          if ((key >> 12) == pre2) {
+            const unsigned slot = atomicAdd(&sm.ncand2, 1u);
+            if (slot < (unsigned)kCand2Cap) { sm.cand2_key[slot] = key; sm.cand2_idx[slot] = (int)lds32(lidx_u32 + c * 4u); }
+          }
+        }
+        settler_sync();
+        const unsigned n2 = sm.ncand2;
+        PROX_TRACE(19);
+        unsigned T, quota;
+        if (n2 <= (unsigned)kCand2Cap) {
+          // rank the few that are left by (score descending, channel ascending)
+          if (tid < (int)n2) {
+            const unsigned key = sm.cand2_key[tid];
+            const int id = sm.cand2_idx[tid];
+            unsigned rank = 0, same_before = 0;
+#pragma unroll 1
+            for (unsigned c = 0; c < n2; ++c) {
+              const unsigned ok = sm.cand2_key[c];
+              const int oi = sm.cand2_idx[c];
+              rank += (ok > key || (ok == key && oi < id)) ? 1u : 0u;
+              same_before += (ok == key && oi < id) ? 1u : 0u;
+            }
+            if (rank == kk2 - 1u) { sm.res[2] = key; sm.res[3] = same_before + 1u; }
+          }
+          settler_sync();
+          T = sm.res[2]; quota = sm.res[3];
+        } else {
+          // many scores agree in their top 20 bits: two more radix steps of 6 bits over the list
+          unsigned prefix = pre2;
+#pragma unroll 1
+          for (int sh = 6; sh >= 0; sh -= 6) {
+            settler_sync();                               // everyone is done with the previous histogram
+            if (tid < 64) sm.hist2[tid] = 0;
+            settler_sync();
+#pragma unroll 1
+            for (unsigned c = tid; c < nb1; c += kSettlers) {
+              const unsigned key = lds32(lkey_u32 + c * 4u);
+              if ((key >> (sh + 6)) == prefix) atomicAdd(&sm.hist2[(key >> sh) & 63u], 1u);
+            }
+            settler_sync();
+            unsigned ab;
+            const unsigned bb = kth_in_segment<2>(sm.hist2, 64, kk2, lane, &ab);
+            prefix = (prefix << 6) | bb;
+            kk2 -= ab;
+          }
+          T = prefix; quota = kk2;
+        }
         PROX_TRACE(20);
-        have_T = true;
+        // ... and keep the block's share of the members above T plus the first `quota` ties at T:
+        // a thread owns a run of the list, counts first (packed in one word), then the places
+        const int ept = ((int)nb1 + kSettlers - 1) / kSettlers;
+        const int c0 = min((int)nb1, tid * ept), c1 = min((int)nb1, c0 + ept);
+        unsigned wt = 0;
+#pragma unroll 1
+        for (int c = c0; c < c1; ++c) {
+          const unsigned key = lds32(lkey_u32 + (uint32_t)c * 4u);
+          wt += ((key > T) ? 1u : 0u) | ((key == T) ? 0x10000u : 0u);
+        }
+        const unsigned inc3 = warp_scan_incl(wt, lane);
+        if (lane == 31) sm.warp_cnt[warp][0] = inc3;
+        settler_sync();
+        {
+          // the totals of the warps in front (every lane reads them itself: the warp may have diverged)
+          unsigned bs = 0;
+#pragma unroll 1
+          for (int w = 0; w < warp; ++w) bs += sm.warp_cnt[w][0];
+          const unsigned ex3 = bs + inc3 - wt;
+          unsigned ra = ex3 & 0xffffu, re = ex3 >> 16;
+#pragma unroll 1
+          for (int c = c0; c < c1; ++c) {
+            const unsigned key = lds32(lkey_u32 + (uint32_t)c * 4u);
+            const bool gt = key > T, eq = key == T;
+            const int pos = (int)(ra + min(re, quota));
+            if ((gt || (eq && re < quota)) && pos >= Rc0 && pos < Rc1) {
+              const int ch = (int)lds32(lidx_u32 + (uint32_t)c * 4u);
+              sm.mysel[ndm + pos - Rc0] = ch;
+              if (p.sel_out) p.sel_out[(int)nd + pos] = ch;
+            }
+            ra += gt ? 1u : 0u; re += eq ? 1u : 0u;
+          }
+        }
+        __threadfence_block();
+        settler_sync();                          // the list is free from here on
+        if (tid == 0) {
+          *reinterpret_cast<volatile int*>(&sm.nready) = n_mine;
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&sm.c_done) = 1;
+        }
+        PROX_TRACE(6);
+        }
       }
-    }
-    if (!have_T) {
-      // Rare (massive ties, e.g. an all-zero input): plain radix refinement over all keys.
-      unsigned prefix = b1;
-      for (int lv = 1; lv < 3; ++lv) {
-        const int sh = (lv == 1) ? 9 : 0, nb = (lv == 1) ? 11 : 9;
+    } else {
+      // No room in shared memory for the keys plus the list of b1's members (a very large
+      // d_ff, or a huge threshold bin such as an all-zero input gives): the whole block
+      // settles the threshold by two radix steps of 10 bits over all keys and keeps its
+      // share of the plain ascending list before the ring starts.
+      const int R0 = (int)(((unsigned)k2 * (unsigned)cta) / (unsigned)G), R1 = (int)(((unsigned)k2 * (unsigned)(cta + 1)) / (unsigned)G);
+      n_mine = min(R1 - R0, kMySelCap);
+      unsigned prefix = b1, kleft = kk;
+#pragma unroll 1
+      for (int sh = 10; sh >= 0; sh -= 10) {
         __syncthreads();
-        for (int i = tid; i < 2048; i += NT) sm.hist[i] = 0;
+        for (int i = tid; i < 1024; i += NT) sm.hist[i] = 0;
         __syncthreads();
+#pragma unroll 1
         for (int i = tid; i < F; i += NT) {
-          const unsigned key = in_smem ? skey[i] : __ldcg(gkey + i);
-          if ((key >> (sh + nb)) == prefix) atomicAdd(&sm.hist[(key >> sh) & ((1u << nb) - 1u)], 1u);
+          const unsigned key = key_at(i);
+          if ((key >> (sh + 10)) == prefix) atomicAdd(&sm.hist[(key >> sh) & 1023u], 1u);
         }
         __syncthreads();
-        if (lv == 1) find_kth_fast<NT, 2048>(sm.hist, kk, sm.wsum, sm.res);
-        else         find_kth_fast<NT, 512>(sm.hist, kk, sm.wsum, sm.res);
-        prefix = (prefix << nb) | sm.res[0];
-        kk -= sm.res[1];
+        unsigned ab;
+        const unsigned bb = kth_in_block<2>(sm.hist, kleft, sm.wsum, lane, warp, &ab);
+        prefix = (prefix << 10) | bb;
+        kleft -= ab;
       }
-      T = prefix; quota = kk;
-    }
-    // Per-chunk counts: the channels above the threshold bin are counted already;
-    // add the candidates that made it (key > T) and note the ties (key == T).
-    bool counted = false;
-    if (have_T && ncand <= (unsigned)kCandCap) {
-      for (unsigned c = tid; c < ncand; c += NT) {
-        const unsigned key = cand_key[c];
-        const int chunk = cand_idx[c] >> 8;
-        if (key > T) atomicAdd(&ccnt[chunk], 1u);
-        else if (key == T) atomicAdd(&ccnt[1024 + chunk], 1u);
-      }
-      counted = true;
-    }
-    auto load8 = [&](int base, unsigned* key) {
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int i = base + hh * 4;
-        uint4 kv = make_uint4(0, 0, 0, 0);
-        if (i < F) kv = in_smem ? *reinterpret_cast<const uint4*>(skey + i)
-                                : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
-        key[hh * 4 + 0] = kv.x; key[hh * 4 + 1] = kv.y; key[hh * 4 + 2] = kv.z; key[hh * 4 + 3] = kv.w;
-      }
-    };
-    if (!counted) {                                        // rare path: count every chunk from the keys
-      for (int q = warp; q < nchk; q += kFusedWarps) {
-        const int base = q * 256 + lane * 8;
-        unsigned key[8];
-        load8(base, key);
-        unsigned cg = 0, ce = 0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const bool in = base + e < F;
-          cg += (in && key[e] > T) ? 1u : 0u;
-          ce += (in && key[e] == T) ? 1u : 0u;
+      const unsigned T = prefix, quota = kleft;
+      __syncthreads();
+      {
+        unsigned cg = 0, ce = 0;                 // separate words: the ties alone may be 65536
+#pragma unroll 1
+        for (int i = i0 + lane; i < i1; i += 32) {
+          const unsigned key = key_at(i);
+          cg += (key > T) ? 1u : 0u; ce += (key == T) ? 1u : 0u;
         }
         cg = __reduce_add_sync(0xffffffffu, cg);
         ce = __reduce_add_sync(0xffffffffu, ce);
-        if (lane == 0) { ccnt[q] = cg; ccnt[1024 + q] = ce; }
+        if (lane == 0) { sm.wsum[warp] = cg; sm.warp_cnt[warp][1] = ce; }
       }
-    }
-    __syncthreads();
-    PROX_TRACE(21);
-    // Ordered compaction: only the chunks whose slice of the ascending list meets
-    // [R0, R1) write anything.
-    for (int q = warp; q < nchk; q += kFusedWarps) {
-      unsigned bg = 0, be = 0;
-      for (int j = lane; j < q; j += 32) { bg += ccnt[j]; be += ccnt[1024 + j]; }
-      bg = __reduce_add_sync(0xffffffffu, bg);
-      be = __reduce_add_sync(0xffffffffu, be);
-      const unsigned cgq = ccnt[q], ceq = ccnt[1024 + q];
-      const int first = (int)(bg + min(be, quota)), end = (int)(bg + cgq + min(be + ceq, quota));
-      if (first >= R1 || end <= R0) continue;              // warp-uniform
-      const int base = q * 256 + lane * 8;
-      unsigned key[8];
-      load8(base, key);
-      unsigned gm = 0, em = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const bool in = base + e < F;
-        gm |= ((in && key[e] > T) ? 1u : 0u) << e;
-        em |= ((in && key[e] == T) ? 1u : 0u) << e;
-      }
-      unsigned rg = bg + lane_prefix8(gm, lt_mask), re = be + lane_prefix8(em, lt_mask);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const bool gt = (gm >> e) & 1u, eq = (em >> e) & 1u;
-        if (gt || (eq && re < quota)) {
-          const int pos = (int)(rg + min(re, quota));
-          if (pos >= R0 && pos < R1) {
-            if (pos - R0 < kMySelCap) sm.mysel[pos - R0] = base + e;
-            if (p.sel_out) p.sel_out[pos] = base + e;
+      __syncthreads();
+      {
+        unsigned bg = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u);
+        unsigned be = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.warp_cnt[lane][1] : 0u);
+        const int first = (int)(bg + min(be, quota));
+        const int end = (int)(bg + sm.wsum[warp] + min(be + sm.warp_cnt[warp][1], quota));
+        if (first < R1 && end > R0) {
+#pragma unroll 1
+          for (int ib = i0; ib < i1; ib += 32) {
+            const int i = ib + lane;
+            const unsigned key = key_at(min(i, F - 1));
+            const bool gt = i < i1 && key > T, eq = i < i1 && key == T;
+            const unsigned mg = __ballot_sync(0xffffffffu, gt), me = __ballot_sync(0xffffffffu, eq);
+            const unsigned myre = be + (unsigned)__popc(me & lt_mask);
+            const int pos = (int)(bg + (unsigned)__popc(mg & lt_mask) + min(myre, quota));
+            if ((gt || (eq && myre < quota)) && pos >= R0 && pos < R0 + n_mine) {
+              sm.mysel[pos - R0] = i;
+              if (p.sel_out) p.sel_out[pos] = i;
+            }
+            bg += (unsigned)__popc(mg); be += (unsigned)__popc(me);
           }
         }
-        rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
       }
+      if (tid == 0) {
+        sm.keys_s0 = sm.keys_s1 = sm.list_s0 = sm.list_s1 = 0;
+        sm.nready = n_mine; sm.keys_done = 1; sm.c_done = 1;
+      }
+      fence_proxy_async();                      // the big buffer becomes a bulk-copy target next
+      __syncthreads();
     }
-    fence_proxy_async();                      // the big buffer becomes a bulk-copy target next
-    __syncthreads();
   }
-  const int n_mine = alive ? min(R1 - R0, kMySelCap) : 0;
 
   PROX_TRACE(5);
   // -------------------------------- D + E: exact gate/up, SwiGLU, masked down
@@ -821,19 +903,38 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       int slot = 0;
       unsigned use = 0;
       bool dead = false;
+      int ready = *reinterpret_cast<volatile int*>(&sm.nready);
+      bool kdone = *reinterpret_cast<volatile int*>(&sm.keys_done) != 0;
+      bool cdone = *reinterpret_cast<volatile int*>(&sm.c_done) != 0;
+      const int ks0 = sm.keys_s0, ks1 = sm.keys_s1, ls0 = sm.list_s0, ls1 = sm.list_s1;
       for (int b0 = 0; b0 < n_mine && !dead; b0 += kChanBatch) {
         const int nb = min(kChanBatch, n_mine - b0);
         for (int q = 0; q < 3 * nb; ++q, ++seq) {
           // A slot always belongs to the same producer: its uses are then armed
           // in program order, so the parity wait below is never two phases behind.
           if (((unsigned)slot & (unsigned)(kFusedProducers - 1)) == pq) {
+            const int mi = b0 + ((q < 2 * nb) ? (q >> 1) : (q - 2 * nb));
+            // The tail of the list (the share of the threshold bin) is written late, and the ring
+            // may not touch the slots under the keys before the consumer warps are done with them.
+            auto blocked = [&]() {
+              return mi >= ready || (!kdone && slot >= ks0 && slot < ks1) || (!cdone && slot >= ls0 && slot < ls1);
+            };
+            if (blocked()) {
+              for (unsigned it = 0; it < kSpinLimit; ++it) {
+                ready = *reinterpret_cast<volatile int*>(&sm.nready);
+                kdone = *reinterpret_cast<volatile int*>(&sm.keys_done) != 0;
+                cdone = *reinterpret_cast<volatile int*>(&sm.c_done) != 0;
+                if (!blocked() || *abortp) break;
+                __nanosleep(64);
+              }
+              if (blocked()) { sm.abort_flag = 1; dead = true; break; }
+            }
             if (use > 0 && !mbar_wait(smem_u32(&sm.mbar_empty[slot]), (use - 1u) & 1u, abortp)) { dead = true; break; }
             const uint16_t* src;
             if (q < 2 * nb) {
-              const int j = sm.mysel[b0 + (q >> 1)];
-              src = ((q & 1) ? p.wu : p.wg) + (size_t)j * D;
+              src = ((q & 1) ? p.wu : p.wg) + (size_t)sm.mysel[mi] * D;
             } else {
-              src = p.wdt + (size_t)sm.mysel[b0 + q - 2 * nb] * D;
+              src = p.wdt + (size_t)sm.mysel[mi] * D;
             }
             const uint32_t bar = smem_u32(&sm.mbar_full[slot]);
             mbar_expect_tx(bar, row_bytes2);
@@ -850,8 +951,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     unsigned base_seq = 0;
     for (int b0 = 0; b0 < n_mine; b0 += kChanBatch) {
       const int nb = min(kChanBatch, n_mine - b0);
-      // D: warp w owns channels w, w+16, ... of the batch
-      for (int c = warp; c < nb; c += kFusedConsumerWarps) {
+      // D: a warp takes the next channel of the batch that nobody has taken yet (the warps
+      // that finish the channel mask join late; rows are consumed in the order they arrive)
+      for (;;) {
+        int c = 0;
+        if (lane == 0) c = (int)atomicAdd(&sm.next_c, 1u);
+        c = __shfl_sync(0xffffffffu, c, 0);
+        if (c >= nb) break;
         const unsigned sq = base_seq + 2u * (unsigned)c;
         const int sg = (int)(sq % (unsigned)NS), su = (int)((sq + 1u) % (unsigned)NS);
         const unsigned ug = sq / (unsigned)NS, uu = (sq + 1u) / (unsigned)NS;
@@ -887,6 +993,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         }
       }
       consumer_sync();
+      if (tid == 0) sm.next_c = 0;               // for the next batch (nobody takes channels during E)
       // E: group gq (TG threads) owns rows gq, gq+NG, ... ; a thread owns EV vectors of y
       {
         const int gq = tid / TG, tg = tid % TG;
@@ -1000,6 +1107,28 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     if (tid == 0) *p.done_ticket = 0;
     __syncthreads();
     PROX_TRACE(9);
+  }
+}
+
+// The persistent kernel lists the kept channels as [definite][share of the
+// threshold bin]; callers of the mask get it in ascending order.  One block:
+// mark the members in a flag array, then an ordered compaction.  Off the hot path.
+__global__ void __launch_bounds__(1024) mask_ascending_kernel(const int* __restrict__ sel, int k2, int F,
+                                                              int* __restrict__ flags, int* __restrict__ out) {
+  __shared__ unsigned long long ws[33];
+  const int tid = threadIdx.x;
+  for (int i = tid; i < F; i += 1024) flags[i] = 0;
+  __syncthreads();
+  for (int i = tid; i < k2; i += 1024) { const int j = sel[i]; if (j >= 0 && j < F) flags[j] = 1; }
+  __syncthreads();
+  unsigned long long run = 0;
+  for (int base = 0; base < F; base += 1024) {
+    const int j = base + tid;
+    const unsigned long long f = (j < F && flags[j]) ? 1ull : 0ull;
+    unsigned long long tot;
+    const unsigned long long ex = block_scan_excl<1024>(f, ws, &tot);
+    if (f && run + ex < (unsigned long long)k2) out[run + ex] = j;
+    run += tot;
   }
 }
 
