@@ -112,6 +112,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+#define PROX_TRACE_AT(k, who) do { if (p.trace && tid == (who)) p.trace[(size_t)cta * 32 + (k)] = global_ns(); } while (0)
 #define PROX_TRACE(k) do { if (p.trace && tid == 0) p.trace[(size_t)cta * 32 + (k)] = global_ns(); } while (0)
 __device__ __forceinline__ void settler_sync() {      // the lower half of the consumer warps
   asm volatile("bar.sync 3, %0;" ::"n"(kSettlers) : "memory");
@@ -197,7 +198,8 @@ __device__ __forceinline__ unsigned kth_in_segment(const unsigned* hist, int top
 // Same over 512 * BPL bins with the whole block (one block barrier inside):
 // warps 0..15 total their segment, then every warp locates the segment and
 // finishes on its own, so the result is in the registers of every thread.
-template <int BPL>
+// CONSUMERS_ONLY: called by the 16 consumer warps alone (named barrier).
+template <int BPL, bool CONSUMERS_ONLY>
 __device__ __forceinline__ unsigned kth_in_block(const unsigned* hist, unsigned k, unsigned* wsum, int lane, int warp,
                                                  unsigned* above) {
   constexpr int NB = 512 * BPL, SEG = 32 * BPL;
@@ -209,7 +211,7 @@ __device__ __forceinline__ unsigned kth_in_block(const unsigned* hist, unsigned 
     s = __reduce_add_sync(0xffffffffu, s);
     if (lane == 0) wsum[warp] = s;
   }
-  __syncthreads();
+  if (CONSUMERS_ONLY) consumer_sync(); else __syncthreads();
   const unsigned v = (lane < 16) ? wsum[lane] : 0u;
   const unsigned inc = warp_scan_incl(v, lane);
   const unsigned ex = inc - v;
@@ -241,6 +243,8 @@ struct FusedSmem {
   unsigned ncand2;
   unsigned prod_seq;       // rows the producers have armed so far (for the give-up path)
   unsigned next_c;         // next channel of the batch to take in the gate/up phase
+  int go;                  // the producer warps may start
+  int n_mine;              // channels of this block (for the producer warps)
   int nready;              // entries of mysel that are final (the definite share first, all of them later)
   int keys_done;           // the consumer warps no longer read the keys near the end of the big buffer
   int c_done;              // ... nor the list of the threshold bin's members
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     mbar_init(smem_u32(&sm.mbar_empty[tid]), kEmptyCount);
     fence_mbar_init();
   }
-  if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; }
+  if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
   if (tid < kMaxSlots) sm.slot_use[tid] = 0;
   {
     const uint4* xg = reinterpret_cast<const uint4*>(p.x);
@@ -306,7 +310,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       __syncthreads();
       PROX_TRACE(10);
       unsigned above1;
-      const unsigned bin1 = kth_in_block<2>(sm.hist, (unsigned)k1, sm.wsum, lane, warp, &above1);
+      const unsigned bin1 = kth_in_block<2, false>(sm.hist, (unsigned)k1, sm.wsum, lane, warp, &above1);
       PROX_TRACE(11);
 #pragma unroll 1
       for (int i = tid; i < D / 2; i += NT) {
@@ -549,6 +553,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   // -------------------------------------------------------------- grid barrier
   // One counter that only grows: a block adds 1 and waits until the count
   // reaches the next multiple of the grid size (no reset, no generation word).
+  fence_proxy_async();                        // phase B's plain accesses to the big buffer come before the ring's bulk copies
   __syncthreads();
   if (tid == 0) {
     __threadfence();                          // cumulative: publishes the block's writes seen through the barrier above
@@ -578,14 +583,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   // is known after two passes over the scores, so its weight rows start to stream
   // while the consumer warps still settle the threshold inside b1.
   int n_mine = 0;
-  if (alive) {
-    // Shared-memory plan: the keys (score bits) sit near the END of the big buffer and the
-    // ascending list of b1's members behind them (before them if it is long): the ring fills
-    // from slot 0 and reaches those slots last.
-    constexpr uint32_t kListFixed = 8192;                  // room for 1024 members behind the keys
-    const bool in_smem = (size_t)F * 4 + kListFixed + 256 <= (size_t)p.big_bytes;
-    const uint32_t list_fixed_off = ((uint32_t)p.big_bytes - kListFixed) & ~127u;
-    const uint32_t key_off = in_smem ? ((list_fixed_off - (uint32_t)F * 4u) & ~127u) : 0u;
+  if (alive && warp < kFusedConsumerWarps) {          // the producer warps wait at the ring for the go flag
+    // Shared-memory plan: the keys (score bits) sit at the END of the big buffer (the ring fills
+    // from slot 0 and reaches those slots last); the ascending list of b1's members goes where
+    // the input index list was (free since phase B), or in front of the keys if it is long.
+    const bool in_smem = (size_t)F * 4 + 256 <= (size_t)p.big_bytes;
+    const uint32_t key_off = in_smem ? (((uint32_t)p.big_bytes - (uint32_t)F * 4u) & ~127u) : 0u;
     const uint32_t skey_u32 = big_u32 + key_off;
     const unsigned* gkey = reinterpret_cast<const unsigned*>(p.scores);
     auto key_at = [&](int i) -> unsigned {
@@ -601,28 +604,33 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     cp_async_commit();
     if (in_smem) {
 #pragma unroll 1
-      for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
+      for (int i = tid; i < F / 4; i += kFusedConsumers) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
     }
     cp_async_commit();
     if (tid < 256) sm.hist2[tid] = 0;
     cp_async_wait<1>();                                    // the histogram (the keys may still be on their way)
-    __syncthreads();
+    consumer_sync();
     PROX_TRACE(16);
     unsigned nd;                                           // channels above bin b1
-    const unsigned b1 = kth_in_block<4>(sm.hist, (unsigned)k2, sm.wsum, lane, warp, &nd);
+    const unsigned b1 = kth_in_block<4, true>(sm.hist, (unsigned)k2, sm.wsum, lane, warp, &nd);
     const unsigned kk = (unsigned)k2 - nd;                 // members of b1 to keep (>= 1)
     const unsigned nb1 = sm.hist[b1];
-    uint32_t list_off = list_fixed_off;
+    uint32_t list_u32 = smem_u32(idx16);                   // 2 * D bytes: room for D / 4 members
+    uint32_t list_off = 0;                                 // offset in the big buffer when it has to go there
+    bool list_in_big = false;
     bool staged = in_smem;                                 // the same in every block
-    if (in_smem && nb1 * 8u > kListFixed) {
-      if ((size_t)nb1 * 8 + 128 <= (size_t)key_off) list_off = (key_off - nb1 * 8u) & ~127u;
-      else staged = false;
+    if (in_smem && (size_t)nb1 * 8 > (size_t)D * 2) {
+      if ((size_t)nb1 * 8 + 128 <= (size_t)key_off) {
+        list_off = (key_off - nb1 * 8u) & ~127u; list_u32 = big_u32 + list_off; list_in_big = true;
+      } else {
+        staged = false;
+      }
     }
-    const int per = ((F + 32 * kFusedWarps - 1) / (32 * kFusedWarps)) * 32;        // channels per warp run (slow path)
+    const int per = ((F + 32 * kFusedConsumerWarps - 1) / (32 * kFusedConsumerWarps)) * 32;        // channels per warp run (slow path)
     const int i0 = min(F, warp * per), i1 = min(F, i0 + per);
     cp_async_wait<0>();
     PROX_TRACE(17);
-    __syncthreads();                                       // the keys are there for everyone; wsum is free again
+    consumer_sync();                                       // the keys are there for everyone; wsum is free again
     if (staged) {
       // k2 * G < 2^31 is checked on the host, so the share bounds fit 32 bits
       const int Rd0 = (int)((nd * (unsigned)cta) / (unsigned)G), Rc0 = (int)((kk * (unsigned)cta) / (unsigned)G);
@@ -650,10 +658,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       if (tid == 0) {
         const uint32_t rb = (uint32_t)D * 2u;
         sm.keys_s0 = (int)(key_off / rb); sm.keys_s1 = (int)((key_off + (uint32_t)F * 4u + rb - 1u) / rb);
-        sm.list_s0 = (int)(list_off / rb); sm.list_s1 = (int)((list_off + nb1 * 8u + rb - 1u) / rb);
-        sm.nready = ndm; sm.keys_done = (ncm == 0) ? 1 : 0; sm.c_done = (ncm == 0) ? 1 : 0;
+        sm.list_s0 = list_in_big ? (int)(list_off / rb) : 0;
+        sm.list_s1 = list_in_big ? (int)((list_off + nb1 * 8u + rb - 1u) / rb) : 0;
+        sm.n_mine = n_mine; sm.nready = ndm; sm.keys_done = (ncm == 0) ? 1 : 0; sm.c_done = (ncm == 0) ? 1 : 0;
       }
-      __syncthreads();
+      consumer_sync();
       PROX_TRACE(18);
       // pass 2: the threads whose definite channels meet the block's share write them out
       const unsigned ex = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u) + inc - cnt;
@@ -678,12 +687,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           }
         }
       }
-      fence_proxy_async();                      // the big buffer becomes a bulk-copy target next
-      __syncthreads();                          // the producer warps leave for the ring here
+      __threadfence_block();
+      consumer_sync();                          // the definite share is listed
+      if (tid == 0) *reinterpret_cast<volatile int*>(&sm.go) = 1;      // the producer warps leave for the ring
       PROX_TRACE(21);
       if (ncm > 0 && warp < kFusedConsumerWarps) {
         // ---- consumer warps only (named barrier): list b1's members in channel order ...
-        const uint32_t lkey_u32 = big_u32 + list_off, lidx_u32 = lkey_u32 + nb1 * 4u;
+        const uint32_t lkey_u32 = list_u32, lidx_u32 = lkey_u32 + nb1 * 4u;
         auto lds32 = [](uint32_t a) -> unsigned { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v; };
         auto sts32 = [](uint32_t a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); };
         if (cnt >> 16) {
@@ -822,22 +832,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       unsigned prefix = b1, kleft = kk;
 #pragma unroll 1
       for (int sh = 10; sh >= 0; sh -= 10) {
-        __syncthreads();
-        for (int i = tid; i < 1024; i += NT) sm.hist[i] = 0;
-        __syncthreads();
+        consumer_sync();
+        for (int i = tid; i < 1024; i += kFusedConsumers) sm.hist[i] = 0;
+        consumer_sync();
 #pragma unroll 1
-        for (int i = tid; i < F; i += NT) {
+        for (int i = tid; i < F; i += kFusedConsumers) {
           const unsigned key = key_at(i);
           if ((key >> (sh + 10)) == prefix) atomicAdd(&sm.hist[(key >> sh) & 1023u], 1u);
         }
-        __syncthreads();
+        consumer_sync();
         unsigned ab;
-        const unsigned bb = kth_in_block<2>(sm.hist, kleft, sm.wsum, lane, warp, &ab);
+        const unsigned bb = kth_in_block<2, true>(sm.hist, kleft, sm.wsum, lane, warp, &ab);
         prefix = (prefix << 10) | bb;
         kleft -= ab;
       }
       const unsigned T = prefix, quota = kleft;
-      __syncthreads();
+      consumer_sync();
       {
         unsigned cg = 0, ce = 0;                 // separate words: the ties alone may be 65536
 #pragma unroll 1
@@ -849,7 +859,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         ce = __reduce_add_sync(0xffffffffu, ce);
         if (lane == 0) { sm.wsum[warp] = cg; sm.warp_cnt[warp][1] = ce; }
       }
-      __syncthreads();
+      consumer_sync();
       {
         unsigned bg = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u);
         unsigned be = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.warp_cnt[lane][1] : 0u);
@@ -872,12 +882,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           }
         }
       }
+      __threadfence_block();
+      consumer_sync();
       if (tid == 0) {
         sm.keys_s0 = sm.keys_s1 = sm.list_s0 = sm.list_s1 = 0;
-        sm.nready = n_mine; sm.keys_done = 1; sm.c_done = 1;
+        sm.n_mine = n_mine; sm.nready = n_mine; sm.keys_done = 1; sm.c_done = 1;
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&sm.go) = 1;
       }
-      fence_proxy_async();                      // the big buffer becomes a bulk-copy target next
-      __syncthreads();
     }
   }
 
@@ -897,7 +909,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   if (warp >= kFusedConsumerWarps) {
     // ---- producer warps: lane 0 of each feeds every kFusedProducers-th slot of
     // the ring (one thread can only start a few million bulk copies a second)
-    if (lane == 0) {
+    if (lane == 0 && alive) {
+      // wait (bounded) until the consumer warps have listed the block's definite share
+      bool go = false;
+      for (unsigned it = 0; it < kSpinLimit; ++it) {
+        if (*reinterpret_cast<volatile int*>(&sm.go)) { go = true; break; }
+        if (*abortp) break;
+        __nanosleep(32);
+      }
+      if (!go) sm.abort_flag = 1;
+      __threadfence_block();
+      fence_proxy_async();                      // the big buffer becomes a bulk-copy target now
+      n_mine = go ? *reinterpret_cast<volatile int*>(&sm.n_mine) : 0;
       const unsigned pq = (unsigned)(warp - kFusedConsumerWarps);
       unsigned seq = 0;
       int slot = 0;
@@ -937,6 +960,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
               src = p.wdt + (size_t)sm.mysel[mi] * D;
             }
             const uint32_t bar = smem_u32(&sm.mbar_full[slot]);
+            if (seq == 0) PROX_TRACE_AT(28, tid);
+            if (seq == 2u * (unsigned)min(n_mine, kChanBatch)) PROX_TRACE_AT(30, tid);
             mbar_expect_tx(bar, row_bytes2);
             bulk_g2s(big_u32 + (uint32_t)slot * row_bytes2, src, row_bytes2, bar);
             atomicMax(&sm.prod_seq, seq + 1u);
