@@ -129,8 +129,13 @@ prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
 /* For B > 1 every token keeps its own masks (the paper covers B = 1 only), and the
  * weights are read once per call for the UNION of the tokens' kept inputs and of
  * their kept channels; a token contributes zero outside its own masks, so its
- * result is the one it would get alone.  prox_ffn_set_union(h, 0) selects the
- * older path that runs the single-token kernels once per token. */
+ * result is the one it would get alone.  With the union, the exact Stage 2
+ * runs as warp-level bf16 tensor-core tiles (16 channels x 8 tokens x 16 inputs)
+ * with fp32 accumulation; in the down projection h enters as a bf16 pair
+ * hi + lo.  prox_ffn_set_union(h, 1) keeps the union but computes with plain fp32
+ * FMAs, prox_ffn_set_union(h, 0) selects the older path that runs the
+ * single-token kernels once per token; any other value (the default) selects the
+ * tensor-core union path. */
 prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on);
 
 /* Launch plan of the persistent kernel for budgets (k1, k2), for diagnostics:

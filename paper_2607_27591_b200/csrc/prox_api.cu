@@ -11,7 +11,7 @@
 
 #include "prox_kernels.cuh"
 #include "prox_fused.cuh"
-#include "prox_batch.cuh"
+#include "prox_batch_mma.cuh"
 
 using namespace prox;
 
@@ -61,6 +61,8 @@ struct prox_ffn {
   float* xu;                // [D][8]  x of every token at a union input (0 if dropped)
   float* member;            // [F][8]  1 / 0 membership of every token at a union channel
   float* hb;                // [F][8]  h of every token at a union channel
+  float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
+  int use_mma;              // batch > 1 Stage 2 runs on the tensor cores
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -298,6 +300,30 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   prox_status_t s;
   if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK)
     return s;
+  const size_t mma_smem = (size_t)8 * (D * 2 + kXPad) + (size_t)kMmaWarps * 256 * sizeof(float);
+  if (h->use_mma && h->gacc && mma_smem <= (size_t)h->smem_optin - 4096) {
+    // tensor-core path: equal ranges of weight units per block, two blocks per SM for gate/up
+    static bool attr_mma = false;
+    if (!attr_mma) {
+      CK(cudaFuncSetAttribute(gateup_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
+      CK(cudaFuncSetAttribute(down_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
+      attr_mma = true;
+    }
+    const int per_sm = (2 * (mma_smem + 1024) <= (size_t)h->smem_optin) ? 2 : 1;
+    {
+      LaunchScope ls(h, kKGateUp, st);
+      gateup_mma_kernel<<<per_sm * h->sm_count, kMmaThreads, mma_smem, st>>>(
+          h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->u_cnt + 1, D, h->gacc);
+      gateup_finish_kernel<<<h->sm_count, 256, 0, st>>>(h->gacc, h->member, h->u_cnt + 1, B, h->hb);
+    }
+    CK(cudaGetLastError());
+    {
+      LaunchScope ls(h, kKDown, st);
+      down_mma_kernel<<<h->sm_count, kMmaThreads, (size_t)kMmaWarps * 512 * sizeof(float), st>>>(
+          h->wdt, h->hb, h->u_ch, h->u_cnt + 1, B, D, h->yacc);
+    }
+    CK(cudaGetLastError());
+  } else {
   const size_t smem = (size_t)B * D * 2;
   static bool attr = false;
   if (!attr) { CK(cudaFuncSetAttribute(gateup_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
@@ -319,6 +345,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
     down_batch_kernel<<<g2, kDownThreads, 0, st>>>(h->wdt, h->hb, h->u_ch, h->u_cnt + 1, B, D, h->yacc);
   }
   CK(cudaGetLastError());
+  }
   const int n = B * D;
   {
     LaunchScope ls(h, kKFinalize, st);
@@ -482,11 +509,14 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
     A(dev_alloc(&h->u_in, (size_t)D)); A(dev_alloc(&h->u_ch, (size_t)F)); A(dev_alloc(&h->u_cnt, (size_t)4));
     A(dev_alloc(&h->xu, (size_t)D * kBT)); A(dev_alloc(&h->member, (size_t)F * kBT));
     A(dev_alloc(&h->hb, (size_t)F * kBT));
+    A(dev_alloc(&h->gacc, (size_t)((F + 15) / 16) * 256));
+    if (st == PROX_OK) A(cudaMemset(h->gacc, 0, (size_t)((F + 15) / 16) * 256 * sizeof(float)));
   }
   A(cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
   A(cudaDeviceGetAttribute(&h->coop, cudaDevAttrCooperativeLaunch, h->device));
   h->use_fused = 1;
   h->use_union = 1;
+  h->use_mma = 1;
   if (st == PROX_OK) A(cudaMemset(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned)));
   A(dev_alloc(reinterpret_cast<uint16_t**>(&h->x_stage), (size_t)MB * D));
   A(dev_alloc(reinterpret_cast<float**>(&h->y_stage), (size_t)MB * D));
@@ -507,7 +537,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
-  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb);
+  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -658,6 +688,7 @@ prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on) {
 prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on) {
   if (!h) return PROX_ERR_INVALID_ARG;
   h->use_union = on != 0;
+  h->use_mma = on != 1;                 // 1 selects the CUDA-core union kernels, any other non-zero value the tensor-core ones
   return PROX_OK;
 }
 
