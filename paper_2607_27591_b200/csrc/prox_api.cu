@@ -62,7 +62,10 @@ struct prox_ffn {
   float* member;            // [F][8]  1 / 0 membership of every token at a union channel
   float* hb;                // [F][8]  h of every token at a union channel
   float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
-  int use_mma;              // batch > 1 Stage 2 runs on the tensor cores
+  int use_mma;              // batch > 1: Stage 2 and the 4-bit proxy GEMM run on the tensor cores
+  float* pacc;              // [F / 64][128 code columns][8] proxy sums of the tensor-core batch path, kept at zero
+  __half* xh;               // [8][D] masked, scaled fp16 x of the tensor-core proxy GEMM
+  float* tokfac;            // [8] per token: what undoes its scaling
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -265,6 +268,25 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   prox_status_t s;
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  const int gshift_m = (h->group == D) ? 31 : 7;
+  if (h->use_mma && h->pacc && h->bits == 4 && F % 64 == 0) {
+    // tensor-core path over all inputs (no union list): masked, scaled fp16 x, then equal ranges
+    // of (strip, K-block) units per block
+    static bool attr_p = false;
+    if (!attr_p) {
+      CK(cudaFuncSetAttribute(proxy_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaWarps * 1024 * (int)sizeof(float)));
+      attr_p = true;
+    }
+    {
+      LaunchScope ls(h, kKProxy, st);
+      proxy_xprep_kernel<<<kBT, 512, 0, st>>>(static_cast<const uint16_t*>(x), h->idx_x, D, k1, B, D, h->xh, h->tokfac);
+      proxy_mma_kernel<<<h->sm_count, kMmaThreads, (size_t)kMmaWarps * 1024 * sizeof(float), st>>>(
+          h->P, h->S, h->xh, h->tokfac, D, F, gshift_m, h->pacc);
+      proxy_mma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
+    }
+    CK(cudaGetLastError());
+    return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
+  }
   if ((s = launch_union(h, h->idx_x, D, nullptr, k1, B, D, x, h->u_in, h->u_cnt, h->xu, st)) != PROX_OK) return s;
   const int ns = nstrips_for(F, h->bits);
   const int nval = 128 * (h->bits == 4 ? 8 : 4);
@@ -510,6 +532,12 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
     A(dev_alloc(&h->xu, (size_t)D * kBT)); A(dev_alloc(&h->member, (size_t)F * kBT));
     A(dev_alloc(&h->hb, (size_t)F * kBT));
     A(dev_alloc(&h->gacc, (size_t)((F + 15) / 16) * 256));
+    {
+      A(dev_alloc(&h->pacc, (size_t)(F / 64) * 1024));
+      if (st == PROX_OK) A(cudaMemset(h->pacc, 0, (size_t)(F / 64) * 1024 * sizeof(float)));
+      A(dev_alloc(&h->xh, (size_t)kBT * D));
+      A(dev_alloc(&h->tokfac, (size_t)kBT));
+    }
     if (st == PROX_OK) A(cudaMemset(h->gacc, 0, (size_t)((F + 15) / 16) * 256 * sizeof(float)));
   }
   A(cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
@@ -537,7 +565,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
-  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc);
+  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
