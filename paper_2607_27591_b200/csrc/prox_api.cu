@@ -64,6 +64,8 @@ struct prox_ffn {
   float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
   int use_mma;              // batch > 1: Stage 2 and the 4-bit proxy GEMM run on the tensor cores
   float* pacc;              // [F / 64][128 code columns][8] proxy sums of the tensor-core batch path, kept at zero
+  unsigned* cmask;          // [F / 4] one byte per channel: which tokens kept it (kept at zero between calls)
+  uint8_t* umask;           // [F] that byte for every union row
   __half* xh;               // [8][D] masked, scaled fp16 x of the tensor-core proxy GEMM
   float* tokfac;            // [8] per token: what undoes its scaling
   void* x_stage;            // device staging for the host-buffer entry point
@@ -320,10 +322,17 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
                                   void* y, cudaStream_t st) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   prox_status_t s;
-  if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK)
-    return s;
   const size_t mma_smem = (size_t)8 * (D * 2 + kXPad) + (size_t)kMmaWarps * 256 * sizeof(float);
-  if (h->use_mma && h->gacc && mma_smem <= (size_t)h->smem_optin - 4096) {
+  const bool mma = h->use_mma && h->gacc && mma_smem <= (size_t)h->smem_optin - 4096;
+  if (mma) {
+    LaunchScope ls(h, kKUnion, st);
+    union_mark_kernel<<<(B * k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B, F, h->cmask, h->dev_status);
+    union_compact_kernel<<<1, 1024, 0, st>>>(h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask);
+    CK(cudaGetLastError());
+  } else if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK) {
+    return s;
+  }
+  if (mma) {
     // tensor-core path: equal ranges of weight units per block, two blocks per SM for gate/up
     static bool attr_mma = false;
     if (!attr_mma) {
@@ -336,7 +345,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
       LaunchScope ls(h, kKGateUp, st);
       gateup_mma_kernel<<<per_sm * h->sm_count, kMmaThreads, mma_smem, st>>>(
           h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->u_cnt + 1, D, h->gacc);
-      gateup_finish_kernel<<<h->sm_count, 256, 0, st>>>(h->gacc, h->member, h->u_cnt + 1, B, h->hb);
+      gateup_finish_kernel<<<h->sm_count, 256, 0, st>>>(h->gacc, h->umask, h->u_cnt + 1, B, h->hb);
     }
     CK(cudaGetLastError());
     {
@@ -536,6 +545,8 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
       A(dev_alloc(&h->pacc, (size_t)(F / 64) * 1024));
       if (st == PROX_OK) A(cudaMemset(h->pacc, 0, (size_t)(F / 64) * 1024 * sizeof(float)));
       A(dev_alloc(&h->xh, (size_t)kBT * D));
+      A(dev_alloc(&h->cmask, (size_t)(F + 3) / 4)); A(dev_alloc(&h->umask, (size_t)F));
+      if (st == PROX_OK) A(cudaMemset(h->cmask, 0, (size_t)((F + 3) / 4) * sizeof(unsigned)));
       A(dev_alloc(&h->tokfac, (size_t)kBT));
     }
     if (st == PROX_OK) A(cudaMemset(h->gacc, 0, (size_t)((F + 15) / 16) * 256 * sizeof(float)));
@@ -565,7 +576,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
-  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac);
+  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->cmask); cudaFree(h->umask);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }

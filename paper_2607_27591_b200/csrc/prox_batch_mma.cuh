@@ -111,17 +111,58 @@ gateup_mma_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__ 
   }
 }
 
+// Union of the tokens' kept channels for the tensor-core path, in two small
+// kernels: every (token, kept channel) sets the token's bit in a byte per channel;
+// one block then lists the channels whose byte is not zero in ascending order,
+// copies the byte next to the list and clears it for the next call.
+__global__ void __launch_bounds__(256)
+union_mark_kernel(const int* __restrict__ lists, int stride, int k, int B, int n, unsigned* __restrict__ mask32,
+                  int* __restrict__ status) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= B * k) return;
+  const int b = i / k, r = i % k;
+  const int id = lists[(size_t)b * stride + r];
+  if (id >= 0 && id < n) atomicOr(mask32 + (id >> 2), (1u << b) << (8 * (id & 3)));
+  else atomicOr(status, kBadChannel);
+}
+
+__global__ void __launch_bounds__(1024)
+union_compact_kernel(unsigned* __restrict__ mask32, int n, int* __restrict__ ulist, int* __restrict__ nu_out,
+                     uint8_t* __restrict__ umask) {
+  __shared__ unsigned long long ws[33];
+  const int tid = threadIdx.x;
+  const int nw = (n + 3) / 4, per = (nw + 1023) / 1024;          // mask words per thread (consecutive)
+  const int w0 = min(nw, tid * per), w1 = min(nw, w0 + per);
+  unsigned cnt = 0;
+  for (int w = w0; w < w1; ++w) {
+    const unsigned m = mask32[w];
+    cnt += ((m & 0xffu) ? 1u : 0u) + ((m & 0xff00u) ? 1u : 0u) + ((m & 0xff0000u) ? 1u : 0u) + ((m >> 24) ? 1u : 0u);
+  }
+  unsigned long long tot;
+  unsigned pos = (unsigned)block_scan_excl<1024>((unsigned long long)cnt, ws, &tot);
+  for (int w = w0; w < w1; ++w) {
+    const unsigned m = mask32[w];
+    mask32[w] = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const unsigned by = (m >> (8 * q)) & 0xffu;
+      if (by && w * 4 + q < n) { ulist[pos] = w * 4 + q; umask[pos] = (uint8_t)by; ++pos; }
+    }
+  }
+  if (tid == 0) *nu_out = (int)tot;
+}
+
 // h[r][b] = SiLU(gate) * up for the tokens that kept channel r, 0 for the others;
 // the accumulator is cleared for the next call.
 __global__ void __launch_bounds__(256)
-gateup_finish_kernel(float* __restrict__ gacc, const float* __restrict__ member, const int* __restrict__ nu_ptr,
+gateup_finish_kernel(float* __restrict__ gacc, const uint8_t* __restrict__ umask, const int* __restrict__ nu_ptr,
                      int B, float* __restrict__ h_out) {
   const int nu = *nu_ptr;
   for (int i = blockIdx.x * 256 + threadIdx.x; i < nu * kBT; i += gridDim.x * 256) {
     const int r = i / kBT, b = i % kBT;
     const float gate = gacc[(size_t)r * 16 + b], up = gacc[(size_t)r * 16 + 8 + b];
     gacc[(size_t)r * 16 + b] = 0.f; gacc[(size_t)r * 16 + 8 + b] = 0.f;
-    h_out[i] = (b < B && member[i] != 0.f) ? up * silu_exact(gate) : 0.f;
+    h_out[i] = (b < B && ((umask[r] >> b) & 1u)) ? up * silu_exact(gate) : 0.f;
   }
 }
 
