@@ -196,14 +196,19 @@ down_mma_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, c
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
     const uint16_t* colp = wdt + (size_t)ct * 64 + g * 8;
-    auto load_unit = [&](int kb, uint4 (&w)[4], float (&hv)[4]) {
+    auto rows_of = [&](int kb, int (&j)[4]) {                  // W_downT rows of the unit's four K slots
+      const int c0 = kb * 16 + 2 * t;
+      const int cr[4] = {c0, c0 + 1, c0 + 8, c0 + 9};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) j[q] = __ldg(ulist + min(cr[q], nu - 1));
+    };
+    auto load_unit = [&](int kb, const int (&j)[4], uint4 (&w)[4], float (&hv)[4]) {
       const int c0 = kb * 16 + 2 * t;
       const int cr[4] = {c0, c0 + 1, c0 + 8, c0 + 9};
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int c = min(cr[q], nu - 1);
-        w[q] = ld_stream(colp + (size_t)ulist[c] * D);
-        hv[q] = (cr[q] < nu) ? __ldg(h + (size_t)c * kBT + g) : 0.f;
+        w[q] = ld_stream(colp + (size_t)j[q] * D);
+        hv[q] = (cr[q] < nu) ? __ldg(h + (size_t)cr[q] * kBT + g) : 0.f;
       }
     };
     auto mma_unit = [&](const uint4 (&w)[4], const float (&hv)[4]) {
@@ -228,12 +233,17 @@ down_mma_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, c
         mma_bf16(acc[2 * q + 1], alo[0], 0u, alo[1], 0u, bo0, bo1);
       }
     };
+    int ja[4], jb[4];
+    if (a + warp < b) rows_of(a + warp, ja);
+    if (a + warp + kMmaWarps < b) rows_of(a + warp + kMmaWarps, jb);
     for (int kb = a + warp; kb < b; kb += 2 * kMmaWarps) {      // two units in flight per warp
       uint4 wa[4], wb[4];
       float ha[4], hb[4];
       const bool two = kb + kMmaWarps < b;
-      load_unit(kb, wa, ha);
-      if (two) load_unit(kb + kMmaWarps, wb, hb);
+      load_unit(kb, ja, wa, ha);
+      if (two) load_unit(kb + kMmaWarps, jb, wb, hb);
+      if (kb + 2 * kMmaWarps < b) rows_of(kb + 2 * kMmaWarps, ja);
+      if (kb + 3 * kMmaWarps < b) rows_of(kb + 3 * kMmaWarps, jb);
       mma_unit(wa, ha);
       if (two) mma_unit(wb, hb);
     }
@@ -347,10 +357,13 @@ proxy_mma_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S, co
       for (int q = 0; q < 4; ++q) { tot[j][q] = 0.f; acc[j][q] = 0.f; }
     corr[0] = corr[1] = corr[2] = corr[3] = 0.f;
     int curg = -1;
+    uint4 s0 = make_uint4(0, 0, 0, 0), s1 = s0;               // scales of the open group (requested when it opened)
+    auto open_group = [&](int grp) {
+      const uint4* sp = reinterpret_cast<const uint4*>(S + (((size_t)grp * nchunks + chunk) * 2 + half) * 16);
+      s0 = __ldg(sp); s1 = __ldg(sp + 1);
+    };
     auto flush = [&](int grp) {
       if (grp < 0) return;
-      const uint4* sp = reinterpret_cast<const uint4*>(S + (((size_t)grp * nchunks + chunk) * 2 + half) * 16);
-      const uint4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
       const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -374,7 +387,7 @@ proxy_mma_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S, co
     };
     auto mma_unit = [&](int kb, const uint2 (&w)[4], const uint2& xp) {
       const int grp = kb >> kbshift;
-      if (grp != curg) { flush(curg); curg = grp; }
+      if (grp != curg) { flush(curg); curg = grp; open_group(grp); }
       const uint32_t A[2] = {w[0].x, w[0].y}, A1[2] = {w[1].x, w[1].y}, Bq[2] = {w[2].x, w[2].y}, B1[2] = {w[3].x, w[3].y};
       uint32_t ue[2], uo[2], ve[2], vo[2];                     // even / odd codes of the row pairs (2t, 2t+1) and (2t+8, 2t+9)
 #pragma unroll
