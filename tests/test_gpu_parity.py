@@ -218,14 +218,14 @@ def test_forward_batched_per_token_masks(pb, toy, B):
 
 @pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0)])
 def test_union_and_per_token_batch_paths_agree(pb, toy, bits, group):
-    """B > 1: one read of the weights for the union of the tokens' masks must give every
-    token the result of the per-token path (and of the oracle)."""
+    """B > 1: one read of the weights for the union of the tokens' masks (on the tensor cores
+    or with plain FMAs) must give every token the result of the per-token path (and of the oracle)."""
     wl, p = toy
     p.quantize(bits, group)
     k1, k2 = wl.points[50]
     B, t0 = 8, 8
     res = []
-    for union in (1, 0):
+    for union in (2, 1, 0):          # tensor-core union kernels, CUDA-core union kernels, one token at a time
         pb.prox_ffn_set_union(p.h, union)
         y = p.y_empty(B)
         m = torch.empty(B, k2, dtype=torch.int32, device="cuda")
@@ -233,7 +233,7 @@ def test_union_and_per_token_batch_paths_agree(pb, toy, bits, group):
         pb.prox_ffn_last_mask(p.h, B, k2, m)
         torch.cuda.synchronize()
         res.append((y.cpu().numpy(), m.cpu().numpy().astype(np.int64)))
-    pb.prox_ffn_set_union(p.h, 1)
+    pb.prox_ffn_set_union(p.h, 2)
     for b in range(B):
         idx, score, sel_ref, thr = p.oracle_stage1(t0 + b, k1, k2)
         for yv, mv in res:
@@ -256,6 +256,33 @@ def test_union_and_per_token_batch_paths_agree(pb, toy, bits, group):
         y_ref, _ = po.stage2(p.x[1 + b], mv, p.wg, p.wu, p.wd)
         assert check_y(y.cpu().numpy()[b], y_ref) < 1e-4
     assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_batch_tokens_of_very_different_magnitude(pb, group):
+    """B = 8 on the tensor-core path: every token's x is scaled by its own power of two before it
+    becomes fp16, so tokens whose magnitudes differ by dozens of binades still get the oracle's masks."""
+    D, F, B = 512, 1024, 8
+    wg, wu, wd, x = inputs.make_small(D, F, B, seed=77)
+    xf = inputs.bf16_bits_to_f32(x).astype(np.float64)
+    for b, e in enumerate((-40, -17, -3, 0, 5, 12, 25, 38)):
+        xf[b] *= 2.0 ** e                              # exact in bf16: only the exponent moves
+    x = inputs.f32_to_bf16_bits(xf.astype(np.float32))
+    p = Problem(pb, wg, wu, wd, x, max_batch=B)
+    try:
+        p.quantize(4, group)
+        k1, k2 = 154, 256
+        _forward_check(pb, p, 0, k1, k2, B=B)
+        sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        sc = torch.empty(B, F, dtype=torch.float32, device="cuda")
+        pb.prox_stage1_mask(p.h, p.t_x, B, k1, k2, sel, sc)
+        torch.cuda.synchronize()
+        for b in range(B):
+            _, score, _, thr = p.oracle_stage1(b, k1, k2)
+            assert float(np.max(np.abs(sc.cpu().numpy()[b] - score)) / thr) < 2e-4
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
 
 
 def test_forward_host_buffers(pb, toy):
