@@ -6,12 +6,19 @@
 //      partials meet through a ticket counter; the last block of a strip writes
 //      the scores |u~ SiLU(g~)| and adds them to a global 2048-bin histogram
 //   -- one grid-wide barrier (bounded spin, self-resetting) --
-//   C  every block: exact k2-th score from the histogram plus a refinement over
-//      the few candidates of the threshold bin; ballot compaction; the block
-//      keeps the slice of the ascending channel list that is its share
+//   C  every block (consumer warps only; the producer warps wait at the ring):
+//      the histogram gives the threshold bin b1; channels in bins above b1 are
+//      kept whatever the exact threshold is.  The kept list is laid out as
+//      [those channels, ascending][kept members of b1, ascending] and block c
+//      owns the c-th share of both parts.  Two passes over the scores list its
+//      share of the first part and the ring starts; half of the consumer warps
+//      then settle the exact threshold inside b1 (ordered list of its members,
+//      8-bit histogram, rank among the few left) and append the block's share
+//      of the second part, while the other half already consumes rows
 //   D  gate/up rows of its channels stream through a shared-memory ring filled
-//      by bulk async copies (cp.async.bulk + mbarrier, four issuing warps); each
-//      consumer warp owns whole channels: h_j = SiLU(x.g_j) (x.u_j)
+//      by bulk async copies (cp.async.bulk + mbarrier, four issuing warps); a
+//      consumer warp takes the next channel nobody has taken:
+//      h_j = SiLU(x.g_j) (x.u_j)
 //   E  the matching rows of channel-major W_down follow in the same ring; warp
 //      groups own whole rows; partial y vectors meet in shared memory and are
 //      added to an fp32 accumulator with vector atomics
