@@ -649,15 +649,26 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       // channels and its members of b1 (packed in one word); one warp scan, warp totals
       const int nq = F / 4, qpt = (nq + kFusedConsumers - 1) / kFusedConsumers;
       const int q0 = min(nq, tid * qpt), q1 = (tid < kFusedConsumers) ? min(nq, q0 + qpt) : q0;
+      // (with up to 64 channels per thread it also keeps them as two bit masks, so that the later
+      // passes walk set bits instead of reading and comparing the scores again)
+      const bool masks = qpt <= 16;
+      unsigned dm[2] = {0u, 0u}, cm[2] = {0u, 0u};           // channels 0..31 and 32..63 of the thread's run
       unsigned cnt = 0;
 #pragma unroll 1
       for (int q = q0; q < q1; ++q) {
         const uint4 kv = key4_at(q * 4);
         const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
+        unsigned d4 = 0, c4 = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const unsigned bin = k4[e] >> 20;
-          cnt += ((bin > b1) ? 1u : 0u) | ((bin == b1) ? 0x10000u : 0u);
+          d4 |= ((bin > b1) ? 1u : 0u) << e;
+          c4 |= ((bin == b1) ? 1u : 0u) << e;
+        }
+        cnt += (unsigned)__popc(d4) | ((unsigned)__popc(c4) << 16);
+        if (masks) {
+          const int rel = q - q0, sh = (rel & 7) * 4;
+          if (rel < 8) { dm[0] |= d4 << sh; cm[0] |= c4 << sh; } else { dm[1] |= d4 << sh; cm[1] |= c4 << sh; }
         }
       }
       const unsigned inc = warp_scan_incl(cnt, lane);
@@ -676,7 +687,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       {
         int dpos = (int)(ex & 0xffffu);
         const int cdef = (int)(cnt & 0xffffu);
-        if (cdef > 0 && dpos < Rd1 && dpos + cdef > Rd0) {
+        if (masks && cdef > 0 && dpos < Rd1 && dpos + cdef > Rd0) {
+#pragma unroll 1
+          for (int hw = 0; hw < 2; ++hw) {
+#pragma unroll 1
+            for (unsigned m = dm[hw]; m; m &= m - 1) {
+              if (dpos >= Rd0 && dpos < Rd1) {
+                const int ch = q0 * 4 + hw * 32 + __ffs((int)m) - 1;
+                sm.mysel[dpos - Rd0] = ch;
+                if (p.sel_out) p.sel_out[dpos] = ch;
+              }
+              ++dpos;
+            }
+          }
+        } else if (cdef > 0 && dpos < Rd1 && dpos + cdef > Rd0) {
 #pragma unroll 1
           for (int q = q0; q < q1; ++q) {
             const uint4 kv = key4_at(q * 4);
@@ -703,7 +727,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         const uint32_t lkey_u32 = list_u32, lidx_u32 = lkey_u32 + nb1 * 4u;
         auto lds32 = [](uint32_t a) -> unsigned { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v; };
         auto sts32 = [](uint32_t a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); };
-        if (cnt >> 16) {
+        if (masks) {
+          unsigned cpos = ex >> 16;
+#pragma unroll 1
+          for (int hw = 0; hw < 2; ++hw) {
+#pragma unroll 1
+            for (unsigned m = cm[hw]; m; m &= m - 1) {
+              const int ch = q0 * 4 + hw * 32 + __ffs((int)m) - 1;
+              if (cpos < nb1) { sts32(lkey_u32 + cpos * 4u, key_at(ch)); sts32(lidx_u32 + cpos * 4u, (unsigned)ch); }
+              ++cpos;
+            }
+          }
+        } else if (cnt >> 16) {
           unsigned cpos = ex >> 16;
 #pragma unroll 1
           for (int q = q0; q < q1; ++q) {
