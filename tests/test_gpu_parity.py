@@ -368,7 +368,9 @@ def test_fused_all_zero_input(pb, toy):
 
 @pytest.mark.parametrize("D,F,k1,k2,bits,group", [
     (16384, 1024, 4915, 239, 4, 128),      # widest d_model the library takes (fused kernel not used: step-wise path)
-    (128, 65536, 38, 15270, 4, 0),         # narrowest d_model, widest d_ff
+    (128, 65536, 38, 15270, 4, 0),         # narrowest d_model, widest d_ff (scores do not fit in shared memory)
+    (128, 65536, 128, 45000, 4, 0),        # ... with more than 256 channels per block (two batches of the ring)
+    (128, 40960, 38, 39000, 4, 128),       # scores in shared memory, more than 256 channels per block
     (8192, 320, 2458, 75, 8, 128),         # ragged last strip, 8-bit codes, two down-projection groups
     (384, 448, 115, 104, 4, 128),          # sizes that are no multiple of the strip or chunk steps
 ])
