@@ -64,6 +64,7 @@ struct prox_ffn {
   float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
   int use_mma;              // batch > 1: Stage 2 and the 4-bit proxy GEMM run on the tensor cores
   float* pacc;              // [F / 64][128 code columns][8] proxy sums of the tensor-core batch path, kept at zero
+  int cmask_marked;         // Stage 1 of the running forward call has set the tokens' bits in cmask already
   unsigned* cmask;          // [F / 4] one byte per channel: which tokens kept it (kept at zero between calls)
   uint8_t* umask;           // [F] that byte for every union row
   __half* xh;               // [8][D] masked, scaled fp16 x of the tensor-core proxy GEMM
@@ -265,30 +266,61 @@ prox_status_t launch_union(prox_ffn* h, const int* lists, int stride, const int*
   return PROX_OK;
 }
 
+// the tensor-core Stage 2 needs x of eight tokens (padded rows) plus a reduction buffer in shared memory
+size_t stage2_mma_smem(const prox_ffn* h) {
+  return (size_t)8 * (h->cfg.d_model * 2 + kXPad) + (size_t)kMmaWarps * 256 * sizeof(float);
+}
+bool stage2_mma_ok(const prox_ffn* h) {
+  return h->use_mma && h->gacc && stage2_mma_smem(h) <= (size_t)h->smem_optin - 4096;
+}
+
+// mark_mask: also set the tokens' bits in the per-channel bytes that the tensor-core Stage 2 of the
+// SAME call turns into the union (only prox_ffn_forward asks for it: the bytes must be consumed)
 prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int k2, int* sel, int sel_stride,
-                                  float* scores, cudaStream_t st) {
+                                  float* scores, cudaStream_t st, bool mark_mask = false) {
+  h->cmask_marked = 0;
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   prox_status_t s;
-  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   const int gshift_m = (h->group == D) ? 31 : 7;
   if (h->use_mma && h->pacc && h->bits == 4 && F % 64 == 0) {
-    // tensor-core path over all inputs (no union list): masked, scaled fp16 x, then equal ranges
-    // of (strip, K-block) units per block
+    // tensor-core path over all inputs (no union list): per-token masked, scaled fp16 x, then equal
+    // ranges of (strip, K-block) units per block, then the per-token channel masks
+    const size_t lim = (size_t)h->smem_optin - 16384;
+    const bool fast_masks = (size_t)D * 2 <= lim && (size_t)F * 4 <= lim;
     static bool attr_p = false;
     if (!attr_p) {
       CK(cudaFuncSetAttribute(proxy_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaWarps * 1024 * (int)sizeof(float)));
+      CK(cudaFuncSetAttribute(batch_input_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
+      CK(cudaFuncSetAttribute(batch_channel_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
       attr_p = true;
+    }
+    if (fast_masks) {
+      LaunchScope ls(h, kKInput, st);
+      batch_input_mask_kernel<<<kBT, kFusedThreads, (size_t)D * 2, st>>>(static_cast<const uint16_t*>(x), B, D, k1,
+                                                                        h->xh, h->tokfac);
+    } else {
+      if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+      LaunchScope ls(h, kKInput, st);
+      proxy_xprep_kernel<<<kBT, 512, 0, st>>>(static_cast<const uint16_t*>(x), h->idx_x, D, k1, B, D, h->xh, h->tokfac);
     }
     {
       LaunchScope ls(h, kKProxy, st);
-      proxy_xprep_kernel<<<kBT, 512, 0, st>>>(static_cast<const uint16_t*>(x), h->idx_x, D, k1, B, D, h->xh, h->tokfac);
       proxy_mma_kernel<<<h->sm_count, kMmaThreads, (size_t)kMmaWarps * 1024 * sizeof(float), st>>>(
           h->P, h->S, h->xh, h->tokfac, D, F, gshift_m, h->pacc);
       proxy_mma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
     }
     CK(cudaGetLastError());
-    return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
+    if (!fast_masks) return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
+    {
+      LaunchScope ls(h, kKChannel, st);
+      batch_channel_mask_kernel<<<B, kFusedThreads, (size_t)F * 4, st>>>(scores, F, k2, sel, sel_stride,
+                                                                        mark_mask ? h->cmask : nullptr);
+    }
+    CK(cudaGetLastError());
+    if (mark_mask) h->cmask_marked = 1;
+    return PROX_OK;
   }
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_union(h, h->idx_x, D, nullptr, k1, B, D, x, h->u_in, h->u_cnt, h->xu, st)) != PROX_OK) return s;
   const int ns = nstrips_for(F, h->bits);
   const int nval = 128 * (h->bits == 4 ? 8 : 4);
@@ -319,14 +351,16 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
 }
 
 prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* sel, int sel_stride, int k2,
-                                  void* y, cudaStream_t st) {
+                                  void* y, cudaStream_t st, bool marked = false) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   prox_status_t s;
-  const size_t mma_smem = (size_t)8 * (D * 2 + kXPad) + (size_t)kMmaWarps * 256 * sizeof(float);
-  const bool mma = h->use_mma && h->gacc && mma_smem <= (size_t)h->smem_optin - 4096;
+  const size_t mma_smem = stage2_mma_smem(h);
+  const bool mma = stage2_mma_ok(h);
   if (mma) {
     LaunchScope ls(h, kKUnion, st);
-    union_mark_kernel<<<(B * k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B, F, h->cmask, h->dev_status);
+    if (!(marked && h->cmask_marked))
+      union_mark_kernel<<<(B * k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B, F, h->cmask, h->dev_status);
+    h->cmask_marked = 0;
     union_compact_kernel<<<1, 1024, 0, st>>>(h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask);
     CK(cudaGetLastError());
   } else if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK) {
@@ -673,8 +707,8 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
   }
   h->sel_unordered = 0;
   if (h->use_union && batch_path_ok(h, B)) {
-    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st)) != PROX_OK) return s;
-    return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st);
+    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
+    return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
   }
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;

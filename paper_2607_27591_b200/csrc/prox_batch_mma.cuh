@@ -20,6 +20,7 @@
 #pragma once
 
 #include "prox_batch.cuh"
+#include "prox_fused.cuh"
 
 namespace prox {
 
@@ -448,6 +449,191 @@ proxy_mma_finish_kernel(float* __restrict__ pacc, int B, int F, float* __restric
     const float gate = *pg, up = *pu;
     *pg = 0.f; *pu = 0.f;
     if (b < B) scores[(size_t)b * F + ch] = fabsf(up * silu_fast(gate));
+  }
+}
+
+// ----------------------------------------------------------------------------
+// Per-token masks of the tensor-core batch path, one 640-thread block per token,
+// built from the selection code of the persistent batch-1 kernel (short loops,
+// thread-owned runs, one warp scan per pass).
+// ----------------------------------------------------------------------------
+
+// Input mask m_x of a token straight into the proxy GEMM's operand: exact top-k1
+// of |x| (ties: lower index first), then xh[b][i] = fp16(x_i * s) at the kept
+// inputs (odd i: x_i * s / 16) and 0 elsewhere, s the power of two that puts max |x| into [2^13, 2^14);
+// tokfac[b] = 2^24 / s.  Token slots beyond B are cleared.
+__global__ void __launch_bounds__(kFusedThreads)
+batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __half* __restrict__ xh,
+                        float* __restrict__ tokfac) {
+  extern __shared__ __align__(16) uint8_t bm_smem[];
+  uint16_t* xs = reinterpret_cast<uint16_t*>(bm_smem);           // [D] bf16 bits of the token
+  __shared__ unsigned hist[1024], hist2[32], wsum[32], smax;
+  constexpr int NT = kFusedThreads;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __half* row = xh + (size_t)b * D;
+  if (b >= B) {
+    for (int i = tid; i < D / 8; i += NT) reinterpret_cast<uint4*>(row)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) tokfac[b] = 16777216.f;
+    return;
+  }
+  if (tid == 0) smax = 0;
+  for (int i = tid; i < 1024 + 32; i += NT) { if (i < 1024) hist[i] = 0; else hist2[i - 1024] = 0; }
+  __syncthreads();
+  unsigned m = 0;
+  for (int i = tid; i < D / 8; i += NT) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + (size_t)b * D) + i);
+    reinterpret_cast<uint4*>(xs)[i] = v;
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) m = max(m, max(w[e] & 0x7fffu, (w[e] >> 16) & 0x7fffu));
+  }
+  m = __reduce_max_sync(0xffffffffu, m);
+  if (lane == 0 && m) atomicMax(&smax, m);
+  __syncthreads();
+  int se = 0;
+  if (smax) se = 13 - ((int)(smax >> 7) - 127);                  // bf16 magnitude bits: exponent in bits 14..7
+  se = max(-100, min(100, se));
+  const float sf = __uint_as_float((unsigned)(se + 127) << 23);
+  if (tid == 0) tokfac[b] = __uint_as_float((unsigned)(24 - se + 127) << 23);
+  const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
+  const bool all = k1 >= D;
+  unsigned T = 0, quota = 0;
+  if (!all) {
+    // level 1: the top 10 of the 15 key bits; level 2: the other 5
+#pragma unroll 1
+    for (int i = tid; i < D / 2; i += NT) {
+      const uint32_t w = xs32[i];
+      atomicAdd(&hist[(w >> 5) & 0x3ffu], 1u);
+      atomicAdd(&hist[(w >> 21) & 0x3ffu], 1u);
+    }
+    __syncthreads();
+    unsigned above1;
+    const unsigned bin1 = kth_in_block<2, false>(hist, (unsigned)k1, wsum, lane, warp, &above1);
+#pragma unroll 1
+    for (int i = tid; i < D / 2; i += NT) {
+      const uint32_t w = xs32[i];
+      const unsigned ka = w & 0x7fffu, kb = (w >> 16) & 0x7fffu;
+      if ((ka >> 5) == bin1) atomicAdd(&hist2[ka & 31u], 1u);
+      if ((kb >> 5) == bin1) atomicAdd(&hist2[kb & 31u], 1u);
+    }
+    __syncthreads();
+    unsigned above2;
+    const unsigned bin2 = kth_in_segment<1>(hist2, 32, (unsigned)k1 - above1, lane, &above2);
+    T = (bin1 << 5) | bin2;
+    quota = (unsigned)k1 - above1 - above2;        // ties at T to accept, lowest index first
+  }
+  // a thread owns a run of 8-input groups; only the ties need their rank (one warp scan + warp totals)
+  const int ngrp = D / 8, gpt = (ngrp + NT - 1) / NT;
+  const int g0 = min(ngrp, tid * gpt), g1 = min(ngrp, g0 + gpt);
+  unsigned ties = 0;
+#pragma unroll 1
+  for (int g = g0; g < g1; ++g) {
+    const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
+    const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ties += (!all && ((w4[e >> 1] >> ((e & 1) * 16)) & 0x7fffu) == T) ? 1u : 0u;
+  }
+  const unsigned inc = warp_scan_incl(ties, lane);
+  __syncthreads();                                 // every warp is done with wsum (k-th search above)
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  unsigned re = __reduce_add_sync(0xffffffffu, (lane < warp) ? wsum[lane] : 0u) + inc - ties;
+#pragma unroll 1
+  for (int g = g0; g < g1; ++g) {
+    const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
+    const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int e2 = 0; e2 < 4; ++e2) {
+      __half hv[2];
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const unsigned bits = (w4[e2] >> (hh * 16)) & 0xffffu, key = bits & 0x7fffu;
+        const bool gt = all || key > T, eq = !all && key == T;
+        const bool keep = gt || (eq && re < quota);
+        re += eq ? 1u : 0u;
+        // odd inputs are the second element of a K-pair, whose code sits four bits higher: x / 16 (exact)
+        hv[hh] = __float2half_rn(keep ? __uint_as_float(bits << 16) * (hh ? sf * 0.0625f : sf) : 0.f);
+      }
+      o[e2] = (uint32_t)__half_as_ushort(hv[0]) | ((uint32_t)__half_as_ushort(hv[1]) << 16);
+    }
+    reinterpret_cast<uint4*>(row)[g] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// Channel mask m_s of a token from its scores: exact top-k2 (ties: lower channel
+// first) by three radix steps over the score bits held in shared memory, then an
+// ordered list of the kept channels; the token's bit is also set in the channel's
+// byte of cmask (the union of the tokens' masks is read off those bytes).
+__global__ void __launch_bounds__(kFusedThreads)
+batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
+                          unsigned* __restrict__ cmask) {
+  extern __shared__ __align__(16) uint8_t bm_smem[];
+  unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
+  __shared__ unsigned hist[2048], wsum[32], wsum2[32];
+  constexpr int NT = kFusedThreads;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned* gkey = reinterpret_cast<const unsigned*>(scores) + (size_t)b * F;
+  const uint32_t skey_u32 = smem_u32(skey);
+  for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
+  cp_async_commit();
+  for (int i = tid; i < 2048; i += NT) hist[i] = 0;
+  cp_async_wait<0>();
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < F; i += NT) atomicAdd(&hist[skey[i] >> 20], 1u);
+  __syncthreads();
+  unsigned ab;
+  unsigned prefix = kth_in_block<4, false>(hist, (unsigned)k2, wsum, lane, warp, &ab);
+  unsigned kleft = (unsigned)k2 - ab;
+#pragma unroll 1
+  for (int sh = 10; sh >= 0; sh -= 10) {           // two more steps of 10 bits
+    __syncthreads();
+    for (int i = tid; i < 1024; i += NT) hist[i] = 0;
+    __syncthreads();
+#pragma unroll 1
+    for (int i = tid; i < F; i += NT) {
+      const unsigned key = skey[i];
+      if ((key >> (sh + 10)) == prefix) atomicAdd(&hist[(key >> sh) & 1023u], 1u);
+    }
+    __syncthreads();
+    const unsigned bb = kth_in_block<2, false>(hist, kleft, wsum, lane, warp, &ab);
+    prefix = (prefix << 10) | bb;
+    kleft -= ab;
+  }
+  const unsigned T = prefix, quota = kleft;
+  // ordered list: a thread owns a run of 4-channel groups
+  const int nq = F / 4, qpt = (nq + NT - 1) / NT;
+  const int q0 = min(nq, tid * qpt), q1 = min(nq, q0 + qpt);
+  unsigned cg = 0, ce = 0;
+#pragma unroll 1
+  for (int q = q0; q < q1; ++q) {
+    const uint4 kv = *reinterpret_cast<const uint4*>(skey + q * 4);
+    const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { cg += (k4[e] > T) ? 1u : 0u; ce += (k4[e] == T) ? 1u : 0u; }
+  }
+  const unsigned ig = warp_scan_incl(cg, lane), ie = warp_scan_incl(ce, lane);
+  __syncthreads();                                 // every warp is done with wsum (k-th search above)
+  if (lane == 31) { wsum[warp] = ig; wsum2[warp] = ie; }
+  __syncthreads();
+  unsigned rg = __reduce_add_sync(0xffffffffu, (lane < warp) ? wsum[lane] : 0u) + ig - cg;
+  unsigned re = __reduce_add_sync(0xffffffffu, (lane < warp) ? wsum2[lane] : 0u) + ie - ce;
+  int* out = sel_out + (size_t)b * sel_stride;
+#pragma unroll 1
+  for (int q = q0; q < q1; ++q) {
+    const uint4 kv = *reinterpret_cast<const uint4*>(skey + q * 4);
+    const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool gt = k4[e] > T, eq = k4[e] == T;
+      if (gt || (eq && re < quota)) {
+        const int ch = q * 4 + e;
+        out[rg + min(re, quota)] = ch;
+        if (cmask) atomicOr(cmask + (ch >> 2), (1u << b) << (8 * (ch & 3)));
+      }
+      rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
+    }
   }
 }
 
