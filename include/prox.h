@@ -144,10 +144,14 @@ prox_status_t prox_ffn_set_union(prox_ffn_t* h, int on);
 prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* info_host);
 
 /* Debug aid: with on != 0 every block of the persistent kernel records time
- * stamps (nanoseconds of the GPU's global timer) per call: slots 0..9 mark the
- * ends of set-up, input mask, proxy GEMV, grid barrier, channel mask, (unused),
- * gate/up + down, partial-y exchange and finalize; slots 10..31 are finer marks
- * inside those phases.  If stamps_host is given, the stamps of the last call are
+ * stamps (nanoseconds of the GPU's global timer) per call.  Slots 0..9: kernel
+ * entry, end of set-up, of the input mask, of the proxy GEMV, of the grid
+ * barrier, of the channel mask (as seen by thread 0, which helps to settle the
+ * threshold bin), slot 6 end of that settling, 7 last row consumed, 8 partial-y
+ * exchange done, 9 finalize done (last block only).  Slots 10..31 are finer
+ * marks inside those phases (16..21: front part of the channel mask, 21 = go
+ * flag for the ring; 28 / 30: first copy / first down-projection row armed by a
+ * producer warp).  If stamps_host is given, the stamps of the last call are
  * copied to it as [min(max_blocks, SM count)][32] uint64 (synchronises).
  * on = 0 frees the buffer. */
 prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int max_blocks);
