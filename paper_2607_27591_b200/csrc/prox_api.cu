@@ -1023,6 +1023,13 @@ prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream
     CK(cudaMemsetAsync(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned), st));
     CK(cudaMemsetAsync(h->ticket, 0, (size_t)h->cfg.max_batch * ns_max * sizeof(unsigned), st));
     CK(cudaMemsetAsync(h->yacc, 0, (size_t)h->cfg.max_batch * h->cfg.d_model * sizeof(float), st));
+    if (h->gacc) {                               // accumulators of the tensor-core batch path (kept at zero between calls)
+      const size_t F = (size_t)h->cfg.d_ff;
+      CK(cudaMemsetAsync(h->gacc, 0, ((F + 15) / 16) * 256 * sizeof(float), st));
+      CK(cudaMemsetAsync(h->pacc, 0, (F / 64) * 1024 * sizeof(float), st));
+      CK(cudaMemsetAsync(h->cmask, 0, ((F + 3) / 4) * sizeof(unsigned), st));
+      h->cmask_marked = 0;
+    }
     CK(cudaStreamSynchronize(st));
   }
   return PROX_OK;
