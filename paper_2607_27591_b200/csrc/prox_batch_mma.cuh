@@ -272,13 +272,12 @@ namespace prox {
 // Stage 1 for B > 1 on the tensor cores (4-bit proxies).
 //
 // A 4-bit code c in the low mantissa bits of an fp16 with a zero exponent field
-// is the subnormal c * 2^-24, exactly; four bits higher it is 16 c * 2^-24.  So
-// two codes of one channel taken from two input rows become an fp16 K-pair with
-// one byte permute and one AND, with no offset to subtract:
-//   u = (rowA & 0x0f0f0f0f) | ((rowB & 0x0f0f0f0f) << 4)     even codes, A low / B high nibble
-//   pair(code 2m) = byte_perm(u, 0, m -> bytes 0 and 2) & 0x00f0000f
-// The factor 16 of the second row is taken out of its x (x / 16 is exact), the
-// 2^-24 and the per-token power-of-two scale of x are undone when a group is
+// is the subnormal c * 2^-24, exactly.  So two codes of one channel taken from
+// two input rows become an fp16 K-pair with one byte permute and no offset to
+// subtract:
+//   ev = row & 0x0f0f0f0f (even codes, one per byte), od = (row >> 4) & 0x0f0f0f0f
+//   pair(code 2m) = bytes (evA[m], 0, evB[m], 0)   (the zero bytes replicate the sign of evA[m])
+// The 2^-24 and the per-token power-of-two scale of x are undone when a group is
 // closed, and the offset binary (c = q + 8) is removed with one more MMA whose A
 // operand is the constant 8: the same sums, the same rounding.
 //
@@ -288,6 +287,12 @@ namespace prox {
 // 64-byte strip.  A K-block never straddles a quantization group (128 inputs), so
 // a warp closes a group by scaling its accumulators.
 // ----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t kpair(uint32_t lo, uint32_t hi, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(lo), "r"(hi), "r"(sel));
+  return d;
+}
+
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -298,8 +303,7 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
 
 // One block per token slot.  The token's kept inputs (its ascending index list)
 // become an fp16 vector over ALL inputs: x * s at a kept input, 0 elsewhere, with
-// s the power of two that puts max |x| into [2^13, 2^14) and odd inputs divided
-// by 16 on top (they are the second element of a K-pair).  With eight tokens the
+// s the power of two that puts max |x| into [2^13, 2^14).  With eight tokens the
 // union of the kept inputs is nearly everything, so the proxy GEMM simply runs
 // over all rows and needs no union list; a dropped input contributes 0 * code.
 // tokfac[b] = 2^24 / s undoes the scaling (and the 2^-24 of the codes).
@@ -326,7 +330,7 @@ proxy_xprep_kernel(const uint16_t* __restrict__ x, const int* __restrict__ idx, 
     for (int r = tid; r < k1; r += 512) {
       const int i = idx[(size_t)b * stride + r];
       const float v = __uint_as_float(((uint32_t)x[(size_t)b * D + i]) << 16) * s;
-      row[i] = __float2half_rn((i & 1) ? v * 0.0625f : v);
+      row[i] = __float2half_rn(v);
     }
   }
 }
@@ -389,24 +393,22 @@ proxy_mma_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S, co
     auto mma_unit = [&](int kb, const uint2 (&w)[4], const uint2& xp) {
       const int grp = kb >> kbshift;
       if (grp != curg) { flush(curg); curg = grp; open_group(grp); }
-      const uint32_t A[2] = {w[0].x, w[0].y}, A1[2] = {w[1].x, w[1].y}, Bq[2] = {w[2].x, w[2].y}, B1[2] = {w[3].x, w[3].y};
-      uint32_t ue[2], uo[2], ve[2], vo[2];                     // even / odd codes of the row pairs (2t, 2t+1) and (2t+8, 2t+9)
+      const uint32_t R[4][2] = {{w[0].x, w[0].y}, {w[1].x, w[1].y}, {w[2].x, w[2].y}, {w[3].x, w[3].y}};
+      uint32_t ev[4][2], od[4][2];                             // even / odd codes of the four rows, one per byte
 #pragma unroll
-      for (int wi = 0; wi < 2; ++wi) {
-        ue[wi] = (A[wi] & 0x0f0f0f0fu) | ((A1[wi] & 0x0f0f0f0fu) << 4);
-        uo[wi] = ((A[wi] >> 4) & 0x0f0f0f0fu) | (A1[wi] & 0xf0f0f0f0u);
-        ve[wi] = (Bq[wi] & 0x0f0f0f0fu) | ((B1[wi] & 0x0f0f0f0fu) << 4);
-        vo[wi] = ((Bq[wi] >> 4) & 0x0f0f0f0fu) | (B1[wi] & 0xf0f0f0f0u);
-      }
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int wi = 0; wi < 2; ++wi) { ev[r][wi] = R[r][wi] & 0x0f0f0f0fu; od[r][wi] = (R[r][wi] >> 4) & 0x0f0f0f0fu; }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int wi = j >> 2;
-        const uint32_t sel = 0x4040u + 0x0101u * (uint32_t)(j & 3);
-        const uint32_t a0 = __byte_perm(ue[wi], 0u, sel) & 0x00f0000fu, a1 = __byte_perm(uo[wi], 0u, sel) & 0x00f0000fu;
-        const uint32_t a2 = __byte_perm(ve[wi], 0u, sel) & 0x00f0000fu, a3 = __byte_perm(vo[wi], 0u, sel) & 0x00f0000fu;
-        mma_f16(acc[j], a0, a1, a2, a3, xp.x, xp.y);
+        const uint32_t m = (uint32_t)(j & 3);
+        // bytes (rowA[m], 0, rowB[m], 0): the zero bytes replicate the sign of rowA[m], which is below 16
+        const uint32_t sel = ((8u | m) << 12) | ((4u + m) << 8) | ((8u | m) << 4) | m;
+        mma_f16(acc[j], kpair(ev[0][wi], ev[1][wi], sel), kpair(od[0][wi], od[1][wi], sel),
+                kpair(ev[2][wi], ev[3][wi], sel), kpair(od[2][wi], od[3][wi], sel), xp.x, xp.y);
       }
-      mma_f16(corr, 0x00800008u, 0x00800008u, 0x00800008u, 0x00800008u, xp.x, xp.y);
+      mma_f16(corr, 0x00080008u, 0x00080008u, 0x00080008u, 0x00080008u, xp.x, xp.y);
     };
     for (int kb = wa; kb < wb; kb += 2) {
       uint2 w0[4], w1[4], xp0, xp1;
@@ -460,7 +462,7 @@ proxy_mma_finish_kernel(float* __restrict__ pacc, int B, int F, float* __restric
 
 // Input mask m_x of a token straight into the proxy GEMM's operand: exact top-k1
 // of |x| (ties: lower index first), then xh[b][i] = fp16(x_i * s) at the kept
-// inputs (odd i: x_i * s / 16) and 0 elsewhere, s the power of two that puts max |x| into [2^13, 2^14);
+// inputs and 0 elsewhere, s the power of two that puts max |x| into [2^13, 2^14);
 // tokfac[b] = 2^24 / s.  Token slots beyond B are cleared.
 __global__ void __launch_bounds__(kFusedThreads)
 batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __half* __restrict__ xh,
@@ -552,8 +554,7 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
         const bool gt = all || key > T, eq = !all && key == T;
         const bool keep = gt || (eq && re < quota);
         re += eq ? 1u : 0u;
-        // odd inputs are the second element of a K-pair, whose code sits four bits higher: x / 16 (exact)
-        hv[hh] = __float2half_rn(keep ? __uint_as_float(bits << 16) * (hh ? sf * 0.0625f : sf) : 0.f);
+        hv[hh] = __float2half_rn(keep ? __uint_as_float(bits << 16) * sf : 0.f);
       }
       o[e2] = (uint32_t)__half_as_ushort(hv[0]) | ((uint32_t)__half_as_ushort(hv[1]) << 16);
     }
