@@ -351,6 +351,31 @@ def test_fused_edge_budgets(pb, toy, k1, k2):
     assert pb.prox_last_device_status(p.h) == 0
 
 
+def test_fused_random_budgets(pb, toy):
+    """Seeded random (k1, k2) pairs, group-128 proxies: the persistent kernel against the oracle."""
+    wl, p = toy
+    p.quantize(4, 128)
+    rng = np.random.default_rng(2024)
+    for _ in range(16):
+        k1 = int(rng.integers(1, p.D + 1))
+        k2 = int(rng.integers(1, p.F + 1))
+        _forward_check(pb, p, int(rng.integers(0, p.x.shape[0])), k1, k2)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+def test_batch_random_budgets(pb, toy):
+    """Seeded random batch sizes and budgets on the tensor-core union path."""
+    wl, p = toy
+    p.quantize(4, 0)
+    rng = np.random.default_rng(7)
+    for _ in range(8):
+        B = int(rng.integers(2, 9))
+        k1 = int(rng.integers(1, p.D + 1))
+        k2 = int(rng.integers(1, p.F + 1))
+        _forward_check(pb, p, int(rng.integers(0, p.x.shape[0] - B + 1)), k1, k2, B=B)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
 def test_fused_all_zero_input(pb, toy):
     """x = 0: every score ties at 0; the mask must be the first k2 channels and y = 0."""
     wl, p = toy
