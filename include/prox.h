@@ -161,9 +161,10 @@ prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int
 prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev, void* stream);
 
 /* Same as prox_ffn_forward with HOST buffers: copies x (host bf16 [B, D]) to
- * the device, runs the path, copies y back and synchronises the stream before
+ * the device, runs the path, brings y back and synchronises the stream before
  * returning.  Pinned host memory makes the copies asynchronous w.r.t. other
- * streams; pageable memory also works. */
+ * streams, and a pinned (mapped) y_host is written by the kernels directly, with
+ * no copy back; pageable memory also works. */
 prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, int k1, int k2,
                                     void* y_host, void* stream);
 

@@ -788,9 +788,20 @@ prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, in
   const size_t D = h->cfg.d_model;
   const size_t ybytes = (size_t)B * D * (h->cfg.out_dtype ? 4 : 2);
   CK(cudaMemcpyAsync(h->x_stage, x_host, (size_t)B * D * 2, cudaMemcpyHostToDevice, st));
-  prox_status_t s = prox_ffn_forward(h, h->x_stage, B, k1, k2, h->y_stage, stream);
+  // If y_host is pinned and mapped, the kernels write the result straight into it (one small
+  // write over the bus by the block that rounds y) and the copy back is not needed.
+  void* y_direct = nullptr;
+  {
+    cudaPointerAttributes pa;
+    if (cudaPointerGetAttributes(&pa, y_host) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer &&
+        aligned16(pa.devicePointer))
+      y_direct = pa.devicePointer;
+    else
+      (void)cudaGetLastError();
+  }
+  prox_status_t s = prox_ffn_forward(h, h->x_stage, B, k1, k2, y_direct ? y_direct : h->y_stage, stream);
   if (s != PROX_OK) return s;
-  CK(cudaMemcpyAsync(y_host, h->y_stage, ybytes, cudaMemcpyDeviceToHost, st));
+  if (!y_direct) CK(cudaMemcpyAsync(y_host, h->y_stage, ybytes, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
   return PROX_OK;
 }
