@@ -375,11 +375,26 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
       attr_mma = true;
     }
     const int per_sm = (2 * (mma_smem + 1024) <= (size_t)h->smem_optin) ? 2 : 1;
+    // whole rows through a ring of bulk copies when 16 of them (a tile) plus a few more fit in shared memory
+    const size_t row_pitch = (size_t)(D * 2 < kGrPiece ? D * 2 : kGrPiece) + 64;
+    int ring_slots = (int)(((size_t)h->smem_optin - 4096 - (size_t)kMmaWarps * 128 * sizeof(float)) / row_pitch);
+    if (ring_slots > kGrMaxSlots) ring_slots = kGrMaxSlots;
     {
       LaunchScope ls(h, kKGateUp, st);
-      gateup_mma_kernel<<<per_sm * h->sm_count, kMmaThreads, mma_smem, st>>>(
-          h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->u_cnt + 1, D, h->gacc);
-      gateup_finish_kernel<<<h->sm_count, 256, 0, st>>>(h->gacc, h->umask, h->u_cnt + 1, B, h->hb);
+      if (D % 512 == 0 && D <= 4096 && ring_slots >= 40) {
+        static bool attr_r = false;
+        if (!attr_r) {
+          CK(cudaFuncSetAttribute(gateup_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
+          attr_r = true;
+        }
+        gateup_rows_kernel<<<h->sm_count, kGrThreads, (size_t)ring_slots * row_pitch + (size_t)kMmaWarps * 128 * sizeof(float), st>>>(
+            h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->umask, h->u_cnt + 1, D, ring_slots, h->hb,
+            h->dev_status);
+      } else {
+        gateup_mma_kernel<<<per_sm * h->sm_count, kMmaThreads, mma_smem, st>>>(
+            h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->u_cnt + 1, D, h->gacc);
+        gateup_finish_kernel<<<h->sm_count, 256, 0, st>>>(h->gacc, h->umask, h->u_cnt + 1, B, h->hb);
+      }
     }
     CK(cudaGetLastError());
     {

@@ -153,6 +153,168 @@ union_compact_kernel(unsigned* __restrict__ mask32, int n, int* __restrict__ uli
   if (tid == 0) *nu_out = (int)tot;
 }
 
+// ----------------------------------------------------------------------------
+// Stage 2a with the weight rows streamed by bulk async copies (d_model <= 4096).
+// Plain loads of rows that are gathered 64 bytes at a time stay near 4.5 TB/s;
+// whole rows through cp.async.bulk, as in the batch-1 kernel, do not.
+// One block per SM: 16 consumer warps + one producer warp whose 32 lanes issue the
+// copies.  A tile is 8 union channels = 16 rows: rows 0..7 of the MMA's A operand
+// are the gate rows, rows 8..15 the up rows of the same channels, so one MMA gives
+// both pre-activations of a channel to the same lane.  A ring slot holds up to 4 KB
+// of a row (+ 64 bytes of padding: the fragment loads of eight rows then fall into
+// different banks); a longer row comes as two sections, so that several tiles are
+// in flight.  A consumer warp owns a sixteenth of every section; its share of x
+// (the B operand) lives in registers for the whole kernel.
+// The warps' partial sums of a tile meet in shared memory and h is written at
+// once: no accumulator in global memory and no finishing kernel.
+// ----------------------------------------------------------------------------
+constexpr int kGrThreads = kMmaThreads + 32;        // 16 consumer warps + one producer warp
+constexpr int kGrMaxSlots = 64;
+constexpr int kGrMaxTiles = 64;                     // tiles of a block whose channels are staged in shared memory
+constexpr int kGrPiece = 4096;                      // bytes of a row in one ring slot (a whole row if it is shorter)
+
+__global__ void __launch_bounds__(kGrThreads, 1)
+gateup_rows_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__ wu,
+                   const uint16_t* __restrict__ x, int B, const int* __restrict__ ulist,
+                   const uint8_t* __restrict__ umask, const int* __restrict__ nu_ptr, int D, int nslots,
+                   float* __restrict__ h_out, int* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t mm_smem[];
+  __shared__ unsigned long long bar_full[kGrMaxSlots / 16], bar_empty[kGrMaxSlots / 16];   // per section of 16 slots
+  __shared__ int abort_flag;
+  __shared__ unsigned n_issued;                                 // sections armed so far (for the give-up path)
+  __shared__ int my_ch[kGrMaxTiles * 8];
+  const int NSEC = nslots / 16;                                 // sections (16 slots) in the ring
+  const uint32_t piece = (uint32_t)min(kGrPiece, D * 2);        // bytes of a row per slot
+  const int nsec = (D * 2) / (int)piece;                        // sections of a row (1 or 2 up to d_model 4096)
+  const uint32_t pitch = piece + 64u;
+  float* red = reinterpret_cast<float*>(mm_smem + (size_t)NSEC * 16 * pitch);     // [16 warps][128]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int nu = *nu_ptr;
+  if (nu <= 0) return;
+  if (tid < NSEC) {
+    mbar_init(smem_u32(&bar_full[tid]), 1);
+    mbar_init(smem_u32(&bar_empty[tid]), kMmaWarps);
+    fence_mbar_init();
+  }
+  if (tid == 0) { abort_flag = 0; n_issued = 0; }
+  const int ntile = (nu + 7) / 8;
+  // the union channels of this block's tiles, so that a producer does not wait for global memory per copy
+  for (int i = tid; i < kGrMaxTiles * 8; i += kGrThreads) {
+    const int tile = blockIdx.x + (i >> 3) * gridDim.x;
+    my_ch[i] = (tile < ntile) ? ulist[min(tile * 8 + (i & 7), nu - 1)] : 0;
+  }
+  fence_proxy_async();
+  __syncthreads();
+  volatile int* abortp = &abort_flag;
+  const uint32_t ring_u32 = smem_u32(mm_smem);
+  if (warp >= kMmaWarps) {
+    // ---- producer warp: one thread starts well under a million copies a second here, so all 32
+    // lanes issue: lanes 0..15 the 16 rows of one section, lanes 16..31 those of the next one.
+    // (One warp, in program order: the use of a slot is always armed after its previous use.)
+    const int per_tile = nsec;                                  // sections per tile
+    const int my_tiles = (ntile - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int nsect = my_tiles * per_tile;                      // sections of this block
+    const int r = lane & 15;
+    bool dead = false;
+    for (int s0 = 0; s0 < nsect && !dead; s0 += 2) {
+      const int si = s0 + (lane >> 4);                          // this lane's section
+      const int ss = si % NSEC;                                 // its place in the ring (16 slots, one barrier pair)
+      const unsigned use = (unsigned)(si / NSEC);
+      bool ok = true;
+      if (si < nsect && use > 0 && r == 0) ok = mbar_wait(smem_u32(&bar_empty[ss]), (use - 1u) & 1u, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { dead = true; break; }
+      if (si < nsect) {
+        const int ti = si / per_tile, sec = si - ti * per_tile;
+        const int tile = (int)blockIdx.x + ti * (int)gridDim.x;
+        const uint32_t bar = smem_u32(&bar_full[ss]);
+        if (r == 0) { mbar_expect_tx(bar, 16u * piece); atomicMax(&n_issued, (unsigned)si + 1u); }
+        __syncwarp();
+        const int ch = (ti < kGrMaxTiles) ? my_ch[ti * 8 + (r & 7)] : ulist[min(tile * 8 + (r & 7), nu - 1)];
+        const uint8_t* src = reinterpret_cast<const uint8_t*>((r < 8 ? wg : wu) + (size_t)ch * D) + (size_t)sec * piece;
+        bulk_g2s(ring_u32 + (uint32_t)(ss * 16 + r) * pitch, src, piece, bar);
+      } else {
+        __syncwarp();
+      }
+    }
+  } else {
+    // ---- consumer warps
+    const int npw = (int)piece / 1024;                          // 32-input pieces of a section per warp (<= 4)
+    uint4 xv[8];                                                // x of token g: sections x pieces of this warp
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int sec = i >> 2, pc = i & 3;
+      xv[i] = make_uint4(0, 0, 0, 0);
+      if (sec < nsec && pc < npw && g < B)
+        xv[i] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)g * D + sec * ((int)piece / 2) + (warp * npw + pc) * 32 + t * 8));
+    }
+    unsigned sidx = 0;                 // running section number of this block
+    bool dead = false;                 // a wait expired: go on without touching the ring, but keep every barrier
+    for (int tile = blockIdx.x; tile < ntile; tile += gridDim.x) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int sec = 0; sec < 2; ++sec) {
+        if (sec < nsec) {
+          // this lane reads the gate row and the up row of channel g of the tile
+          const int ss = (int)(sidx % (unsigned)NSEC);
+          const int sg = ss * 16 + g, su = ss * 16 + 8 + g;
+          // One thread alone waits for the 16 rows of the section: hundreds of threads polling the
+          // barrier slow the copies down.  The others learn of it at a block barrier.
+          if (tid == 0 && !dead) {
+            if (!mbar_wait(smem_u32(&bar_full[ss]), (sidx / (unsigned)NSEC) & 1u, abortp)) abort_flag = 1;
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory");
+          if (*abortp) dead = true;
+          if (!dead) {
+            const uint32_t pg = ring_u32 + (uint32_t)sg * pitch + (uint32_t)(warp * npw) * 64u + (uint32_t)t * 16u;
+            const uint32_t pu = ring_u32 + (uint32_t)su * pitch + (uint32_t)(warp * npw) * 64u + (uint32_t)t * 16u;
+#pragma unroll
+            for (int pc = 0; pc < 4; ++pc) {
+              if (pc < npw) {
+                const uint4 gl = lds128(pg + (uint32_t)pc * 64u), ul = lds128(pu + (uint32_t)pc * 64u);
+                const uint4 xw = xv[sec * 4 + pc];
+                mma_bf16(acc, gl.x, ul.x, gl.y, ul.y, xw.x, xw.y);
+                mma_bf16(acc, gl.z, ul.z, gl.w, ul.w, xw.z, xw.w);
+              }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_n(smem_u32(&bar_empty[ss]), 1u);       // this warp is done with the section
+          }
+          ++sidx;
+        }
+      }
+      // the warps' partial sums meet: [gate | up][channel g][token]
+      float* mine = red + warp * 128;
+      mine[g * 8 + 2 * t] = acc[0]; mine[g * 8 + 2 * t + 1] = acc[1];
+      mine[64 + g * 8 + 2 * t] = acc[2]; mine[64 + g * 8 + 2 * t + 1] = acc[3];
+      asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory");
+      if (tid < 64) {
+        float gate = 0.f, up = 0.f;
+#pragma unroll
+        for (int w = 0; w < kMmaWarps; ++w) { gate += red[w * 128 + tid]; up += red[w * 128 + 64 + tid]; }
+        const int r = tile * 8 + (tid >> 3), b = tid & 7;
+        if (r < nu) h_out[(size_t)r * kBT + b] = (b < B && ((umask[r] >> b) & 1u)) ? up * silu_exact(gate) : 0.f;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kMmaThreads) : "memory");
+    }
+  }
+  __syncthreads();
+  if (abort_flag && tid == 0) {
+    // a wait expired: the copies that were armed last may still be on their way; wait for them
+    // (bounded) so that none lands after the block has left
+    atomicOr(status, kWaitExpired);
+    const unsigned issued = n_issued;                           // sections armed
+    const unsigned first = issued > (unsigned)NSEC ? issued - (unsigned)NSEC : 0u;
+    for (unsigned q = first; q < issued; ++q) {
+      const uint32_t bar = smem_u32(&bar_full[q % (unsigned)NSEC]);
+      for (unsigned it = 0; it < 8192u; ++it) {
+        if (mbar_try_wait(bar, (q / (unsigned)NSEC) & 1u)) break;
+        __nanosleep(256);
+      }
+    }
+  }
+}
+
 // h[r][b] = SiLU(gate) * up for the tokens that kept channel r, 0 for the others;
 // the accumulator is cleared for the next call.
 __global__ void __launch_bounds__(256)
