@@ -22,7 +22,9 @@ library SiLU; Stage 2 against the dense FFN with unselected channels zeroed;
 exact-score mask against a full sort; the allocation tables printed in the
 paper; the paper's closed forms q_Lap, q_G, eta, Corr; the residual bound
 ||xW - x_sp W|| <= ||r|| ||W||; the order-preservation condition; quantizer
-invariants; a hand-worked 4x4 example.  The mask and output *values* on random
+invariants; a hand-worked 4x4 example; the ablation forms against the dense FFN
+(all inputs and channels kept, original weights as proxy) and against Stage 2 on
+the exact top-k of |s|.  The mask and output *values* on random
 inputs have no worked example in the paper: parity unpinned for those beyond
 the properties above.
 """
@@ -34,7 +36,7 @@ __all__ = [
     "bf16_to_f64", "f64_to_bf16_bits", "silu", "dense_ffn", "quantize_proxy",
     "dequantize", "input_topk", "input_threshold", "input_sparse_projection", "proxy_scores", "channel_topk",
     "channel_threshold", "stage2", "forward", "forward_batch", "allocate_budget",
-    "sparsity_to_k", "effective_sparsity",
+    "sparsity_to_k", "effective_sparsity", "proxy_values", "forward_proxy_values",
 ]
 
 
@@ -203,6 +205,33 @@ def forward(x, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down):
     sel, thr = channel_topk(score, k2)
     y, s_sp = stage2(x, sel, w_gate, w_up, w_down)
     return {"idx_x": idx_x, "score": score, "sel": sel, "threshold": thr, "y": y, "s_sp": s_sp}
+
+
+# ------------------------------------------------------------ ablation forms
+def proxy_values(x, idx_x, deq_gate, deq_up) -> np.ndarray:
+    """The signed proxy intermediate state s~ = u~ (.) h~ of Sec. 4.1 (its
+    magnitude is what `proxy_scores` ranks)."""
+    u_t = input_sparse_projection(x, idx_x, deq_up)
+    h_t = silu(input_sparse_projection(x, idx_x, deq_gate))
+    return u_t * h_t
+
+
+def forward_proxy_values(x, k1: int, k2: int, deq_gate, deq_up, w_down):
+    """Ablation A3 of Sec. "Ablation Studies" (necessity of exact computation):
+    everything as in Prox, but Stage 2's exact gate/up is skipped and the
+    selected proxy values themselves enter the down projection,
+        y = Pi_in(s~, W_down, m_s).
+    With the original weights passed as the proxy this is the execution pattern
+    the paper attributes to TEAL (Sec. 2.2): input sparsity on x for gate/up,
+    then input sparsity on the resulting s for the down projection.  (The
+    ablation with 16-bit proxies, A1, needs no function of its own: pass the
+    original weights as `deq_gate`, `deq_up` to `forward`.)"""
+    idx_x = input_topk(x, k1)
+    s_t = proxy_values(x, idx_x, deq_gate, deq_up)
+    score = np.abs(s_t)
+    sel, thr = channel_topk(score, k2)
+    y = np.asarray(w_down)[:, sel].astype(np.float64) @ s_t[sel]
+    return {"idx_x": idx_x, "score": score, "sel": sel, "threshold": thr, "y": y, "s_sp": s_t[sel]}
 
 
 def forward_batch(xs, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down):

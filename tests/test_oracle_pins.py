@@ -435,3 +435,64 @@ def test_batch_tokens_are_independent():
     for t, o in enumerate(outs):
         single = po.forward(x[t], 77, 100, dg, du, wg, wu, wd)
         assert np.array_equal(o["y"], single["y"]) and np.array_equal(o["sel"], single["sel"])
+
+
+# ------------------------------------------------------------ ablation forms
+def test_proxy_values_into_down_with_exact_proxy_and_nothing_dropped_is_dense():
+    """A3 form with the original weights as proxy, k1 = d_model, k2 = d_ff: the
+    proxy state is the exact s, so y is the dense FFN (Sec. 2.1) by library ops."""
+    wg, wu, wd, x = _problem(seed=11)
+    d_model, d_ff = wg.shape[1], wg.shape[0]
+    for t in range(x.shape[0]):
+        out = po.forward_proxy_values(x[t], d_model, d_ff, wg, wu, wd)
+        xt = torch.from_numpy(x[t])
+        y_ref = torch.from_numpy(wd) @ ((torch.from_numpy(wu) @ xt) *
+                                        torch.nn.functional.silu(torch.from_numpy(wg) @ xt))
+        np.testing.assert_allclose(out["y"], y_ref.numpy(), rtol=1e-10, atol=1e-13)
+
+
+def test_input_then_state_sparsity_pattern_by_library_ops():
+    """The pattern the paper attributes to TEAL (Sec. 2.2): zero all but the k1
+    largest |x|, run gate/up densely on that x (library matmul), zero all but the
+    k2 largest |s|, run the down projection densely.  Written here with masks and
+    torch ops, not with the oracle's gathers."""
+    wg, wu, wd, x = _problem(seed=12)
+    d_model, d_ff = wg.shape[1], wg.shape[0]
+    k1, k2 = 90, 130
+    for t in range(x.shape[0]):
+        out = po.forward_proxy_values(x[t], k1, k2, wg, wu, wd)
+        order = np.argsort(-np.abs(x[t]), kind="stable")[:k1]
+        mx = np.zeros(d_model)
+        mx[order] = 1.0
+        xs = torch.from_numpy(x[t] * mx)
+        s = (torch.from_numpy(wu) @ xs) * torch.nn.functional.silu(torch.from_numpy(wg) @ xs)
+        keep = np.argsort(-np.abs(s.numpy()), kind="stable")[:k2]
+        ms = np.zeros(d_ff)
+        ms[keep] = 1.0
+        y_ref = torch.from_numpy(wd) @ (s * torch.from_numpy(ms))
+        assert np.array_equal(out["sel"], np.sort(keep))
+        np.testing.assert_allclose(out["y"], y_ref.numpy(), rtol=1e-9, atol=1e-13)
+
+
+def test_proxy_values_have_the_sign_that_scores_drop():
+    wg, wu, wd, x = _problem(seed=13)
+    dg = po.dequantize(*po.quantize_proxy(wg, 4, 0), 0)
+    du = po.dequantize(*po.quantize_proxy(wu, 4, 0), 0)
+    idx = po.input_topk(x[0], 64)
+    v = po.proxy_values(x[0], idx, dg, du)
+    assert np.array_equal(np.abs(v), po.proxy_scores(x[0], idx, dg, du))
+    assert (v < 0).any() and (v > 0).any()
+    # on a hand-made case: u~ = -2, g~ = 1  ->  s~ = -2 * SiLU(1)
+    w_g = np.array([[1.0, 0.0]])
+    w_u = np.array([[-2.0, 5.0]])
+    s = po.proxy_values(np.array([1.0, 0.25]), np.array([0]), w_g, w_u)
+    assert s[0] == pytest.approx(-2.0 / (1.0 + math.exp(-1.0)), rel=1e-15)
+
+
+def test_sixteen_bit_proxy_budget_uses_unit_cost_ratio():
+    """A1 reallocates the two stages for a 16-bit proxy: alpha = 1 in the cost
+    model of Sec. 4.2, e = s2 - 2 alpha (1 - s1) / 3."""
+    for e in (0.4, 0.5, 0.6, 0.7):
+        s1, s2 = po.allocate_budget(e, alpha=1.0)
+        assert 0.0 <= s1 <= 1.0 and 0.0 <= s2 <= 1.0
+        assert po.effective_sparsity(s1, s2, alpha=1.0) == pytest.approx(e, abs=1e-12)
