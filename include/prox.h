@@ -91,6 +91,12 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate_d
  * ([d_ff, d_model], Sec. 3.1: y = sum_j s_j W_down[j,:]) so that the masked
  * down projection reads one contiguous row per kept channel.
  * bits in {4, 8}; group_size in {0, 128}.  May be called again to re-pack.
+ * bits = 16 (group_size 0 only) stores the original bf16 weights themselves in
+ * the same input-major order, with no scales: the 16-bit proxy of ablation A1
+ * (Sec. "Ablation Studies"), and the 16-bit input-sparse GEMV that the cost
+ * ratio alpha of Sec. 4.2 compares the integer proxy GEMV with.  With 16-bit
+ * proxies the forward calls take the step-wise kernels (the fused kernel and
+ * the batched Stage 1 read integer codes); prox_proxy_export is UNSUPPORTED.
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA, OOM. */
 prox_status_t prox_quantize_proxy(prox_ffn_t* h, int bits, int group_size, void* stream);
 
@@ -218,6 +224,17 @@ prox_status_t prox_stage2_ffn_var(prox_ffn_t* h, const void* x_dev, int B, const
                                   const int32_t* count_dev, void* y_dev, void* stream);
 prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x_dev, int B, float tau_x,
                                          float tau_s, void* y_dev, void* stream);
+
+/* Ablation A3 of Sec. "Ablation Studies" (necessity of exact computation):
+ * Stage 1 as in prox_ffn_forward, then the signed proxy values
+ * s~_j = u~_j SiLU(g~_j) of the k2 selected channels enter the down projection,
+ *     y = sum_{j in m_s} s~_j W_down[j,:],
+ * and the exact gate/up of Stage 2 is skipped.  With 16-bit proxies this is the
+ * pattern Sec. 2.2 attributes to TEAL: input sparsity on x for gate/up, then
+ * input sparsity on the resulting s for the down projection.
+ * Arguments, layouts and errors as prox_ffn_forward; step-wise kernels. */
+prox_status_t prox_ffn_forward_proxy_values(prox_ffn_t* h, const void* x_dev, int B, int k1, int k2,
+                                            void* y_dev, void* stream);
 
 /* Runtime mask counts accumulated by the threshold entry points since the last
  * reset (appendix "Threshold Calibration and Runtime Sparsity":

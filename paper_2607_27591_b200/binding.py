@@ -52,6 +52,7 @@ _SIGS = {
     "prox_stage1_mask_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp, _vp, _vp],
     "prox_stage2_ffn_var": [_vp, _vp, _i, _vp, _vp, _vp, _vp],
     "prox_ffn_forward_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp],
+    "prox_ffn_forward_proxy_values": [_vp, _vp, _i, _i, _i, _vp, _vp],
     "prox_runtime_sparsity": [_vp, _d, C.POINTER(C.c_int64), C.POINTER(_d), C.POINTER(_d), C.POINTER(_d), _i],
     "prox_allocate_budget": [_d, _d, _d, _d, _d, C.POINTER(_d), C.POINTER(_d)],
     "prox_sparsity_to_k": [_d, _i, C.POINTER(_i)],
@@ -195,6 +196,11 @@ def prox_stage2_ffn_var(handle: int, x, B: int, sel, count, y, stream=None) -> N
 def prox_ffn_forward_threshold(handle: int, x, B: int, tau_x: float, tau_s: float, y, stream=None) -> None:
     _check(_lib.prox_ffn_forward_threshold(handle, _ptr(x), B, tau_x, tau_s, _ptr(y), _ptr(stream)),
            "prox_ffn_forward_threshold")
+
+
+def prox_ffn_forward_proxy_values(handle: int, x, B: int, k1: int, k2: int, y, stream=None) -> None:
+    _check(_lib.prox_ffn_forward_proxy_values(handle, _ptr(x), B, k1, k2, _ptr(y), _ptr(stream)),
+           "prox_ffn_forward_proxy_values")
 
 
 def prox_runtime_sparsity(handle: int, alpha: float = 1.0 / 3.0, reset: bool = False):

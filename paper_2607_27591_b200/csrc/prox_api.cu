@@ -41,6 +41,7 @@ struct prox_ffn {
   size_t part_floats;
   unsigned* ticket;         // [maxB][nstrips_max]
   float* scores;            // [maxB][F]
+  float* svals;             // [maxB][F] signed proxy values (proxy-values-into-down variant), on first use
   int* sel;                 // [maxB][F]
   int* cnt_s;               // [maxB]
   float* hbuf;              // [maxB][F]
@@ -95,7 +96,7 @@ prox_status_t map_cuda(cudaError_t e) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int ch_per_chunk(int bits) { return bits == 4 ? 16 : 8; }
+int ch_per_chunk(int bits) { return bits == 4 ? 16 : (bits == 8 ? 8 : 4); }
 
 template <typename T>
 cudaError_t dev_alloc(T** p, size_t count) {
@@ -177,7 +178,7 @@ prox_status_t launch_input_select(prox_ffn* h, const void* x, int B, int k1, flo
 }
 
 prox_status_t launch_proxy(prox_ffn* h, const void* x, int B, const int* idx, int stride,
-                           const int* cnt, int k1, float* scores, cudaStream_t st) {
+                           const int* cnt, int k1, float* scores, cudaStream_t st, float* values = nullptr) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   const int ns = nstrips_for(F, h->bits);
   const int ks = ksplit_for(h, B, k1);
@@ -190,12 +191,17 @@ prox_status_t launch_proxy(prox_ffn* h, const void* x, int B, const int* idx, in
     const size_t smem = (size_t)kProxyWarps * ProxyFmt<4>::NACC * 32 * sizeof(float);
     proxy_gemv_kernel<4><<<grid, kProxyThreads, smem, st>>>(
         h->P, h->S, static_cast<const uint16_t*>(x), idx, stride, cnt, k1, D, F, gshift, h->part,
-        h->ticket, scores, h->dev_status);
-  } else {
+        h->ticket, scores, values, h->dev_status);
+  } else if (h->bits == 8) {
     const size_t smem = (size_t)kProxyWarps * ProxyFmt<8>::NACC * 32 * sizeof(float);
     proxy_gemv_kernel<8><<<grid, kProxyThreads, smem, st>>>(
         h->P, h->S, static_cast<const uint16_t*>(x), idx, stride, cnt, k1, D, F, gshift, h->part,
-        h->ticket, scores, h->dev_status);
+        h->ticket, scores, values, h->dev_status);
+  } else {
+    const size_t smem = (size_t)kProxyWarps * ProxyFmt<16>::NACC * 32 * sizeof(float);
+    proxy_gemv_kernel<16><<<grid, kProxyThreads, smem, st>>>(
+        h->P, h->S, static_cast<const uint16_t*>(x), idx, stride, cnt, k1, D, F, gshift, h->part,
+        h->ticket, scores, values, h->dev_status);
   }
   CK(cudaGetLastError());
   return PROX_OK;
@@ -211,6 +217,9 @@ prox_status_t launch_channel_select(prox_ffn* h, const float* scores, int B, int
   return PROX_OK;
 }
 
+prox_status_t launch_down(prox_ffn* h, int B, const int* sel, int stride, const int* cnt, int k2, void* y,
+                          cudaStream_t st);
+
 prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, int stride,
                             const int* cnt, int k2, void* y, cudaStream_t st) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
@@ -223,6 +232,12 @@ prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, i
         h->dev_status);
   }
   CK(cudaGetLastError());
+  return launch_down(h, B, sel, stride, cnt, k2, y, st);
+}
+
+prox_status_t launch_down(prox_ffn* h, int B, const int* sel, int stride, const int* cnt, int k2, void* y,
+                          cudaStream_t st) {
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
   const int dtiles = (D + kDownThreads * 8 - 1) / (kDownThreads * 8);
   int nsplit = (2 * h->sm_count + dtiles * B - 1) / (dtiles * B);
   if (nsplit > k2) nsplit = k2;
@@ -243,8 +258,9 @@ prox_status_t launch_stage2(prox_ffn* h, const void* x, int B, const int* sel, i
 }
 
 // ---- batch > 1: union path -----------------------------------------------------
-bool batch_path_ok(const prox_ffn* h, int B) {
+bool batch_path_ok(const prox_ffn* h, int B, bool stage1 = false) {
   if (B < 2 || !h->u_in) return false;
+  if (stage1 && h->bits == 16) return false;             // the batch Stage 1 reads integer proxies
   const size_t xs_bytes = (size_t)B * h->cfg.d_model * 2;
   const size_t red_bytes = (size_t)4 * kBT * 128 * (h->bits == 4 ? 8 : 4) * sizeof(float);
   const size_t ubits = (size_t)(B + 2) * ((h->cfg.d_ff + 31) / 32) * 4;
@@ -446,7 +462,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   FusedPlan pl;
   std::memset(&pl, 0, sizeof(pl));
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
-  if (!h->use_fused || !h->coop) return pl;
+  if (!h->use_fused || !h->coop || h->bits == 16) return pl;       // the fused kernel reads integer proxies
   const int G = h->sm_count;
   const size_t fixed = ((sizeof(FusedSmem) + 127) & ~size_t(127)) + (size_t)8 * D;   // + x bf16, idx, x fp32
   if ((size_t)h->smem_optin < fixed + (size_t)6 * D + 16384) return pl;
@@ -623,7 +639,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   if (!h) return;
   free_packed(h);
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
-  cudaFree(h->scores); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
+  cudaFree(h->scores); cudaFree(h->svals); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
   cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->cmask); cudaFree(h->umask);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
@@ -636,14 +652,25 @@ void prox_ffn_destroy(prox_ffn_t* h) {
 
 prox_status_t prox_quantize_proxy(prox_ffn_t* h, int bits, int group_size, void* stream) {
   if (!h) return PROX_ERR_INVALID_ARG;
-  if (bits != 4 && bits != 8) return PROX_ERR_UNSUPPORTED;
+  if (bits != 4 && bits != 8 && bits != 16) return PROX_ERR_UNSUPPORTED;
   if (group_size != 0 && group_size != 128) return PROX_ERR_UNSUPPORTED;
+  if (bits == 16 && group_size != 0) return PROX_ERR_UNSUPPORTED;   // 16-bit proxies are the weights: no scales
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   const int G = group_size == 0 ? D : group_size;
   prox_status_t s = alloc_packed(h, bits, G);
   if (s != PROX_OK) { free_packed(h); return s; }
   const int ngroups = D / G;
+  if (bits == 16) {
+    const long long total = (long long)(F / 4) * 4 * D;
+    const int bs = 256;
+    CK(cudaMemsetAsync(h->S, 0, h->s_count * sizeof(__half), st));
+    CK(cudaMemsetAsync(h->s_plain, 0, (size_t)2 * F * ngroups * sizeof(float), st));
+    proxy_pack16_kernel<<<(unsigned)((total + bs - 1) / bs), bs, 0, st>>>(h->wg, h->wu, D, F,
+                                                                         reinterpret_cast<uint32_t*>(h->P));
+    h->launches++;
+    CK(cudaGetLastError());
+  } else {
   {
     const long long warps = 2ll * F * ngroups;
     const long long threads = warps * 32;
@@ -662,6 +689,7 @@ prox_status_t prox_quantize_proxy(prox_ffn_t* h, int bits, int group_size, void*
         F, G, bits, h->s_plain, reinterpret_cast<uint32_t*>(h->P));
     h->launches++;
     CK(cudaGetLastError());
+  }
   }
   {
     dim3 grid((F + 31) / 32, (D + 31) / 32), block(32, 8);
@@ -690,7 +718,7 @@ prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x, int B, int k1, int 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model;
   float* sc = scores ? scores : h->scores;
-  if (h->use_union && batch_path_ok(h, B)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st);
+  if (h->use_union && batch_path_ok(h, B, true)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st);
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, sc, st)) != PROX_OK) return s;
   return launch_channel_select(h, sc, B, k2, 0.f, 0, sel, k2, nullptr, st);
@@ -721,14 +749,43 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
     if (pl.ok) { h->sel_unordered = 1; return launch_fused(h, pl, x, k1, k2, y, h->sel, st); }
   }
   h->sel_unordered = 0;
-  if (h->use_union && batch_path_ok(h, B)) {
+  if (h->use_union && batch_path_ok(h, B, true)) {
     if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
     return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
   }
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
   if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
+  if (h->use_union && batch_path_ok(h, B)) return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, false);
   return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
+}
+
+// Ablation A3 of Sec. "Ablation Studies": Stage 1 as always, then the selected proxy values themselves
+// enter the down projection (no exact gate/up).  With 16-bit proxies this is the input-sparse /
+// state-sparse pattern of Sec. 2.2.
+prox_status_t prox_ffn_forward_proxy_values(prox_ffn_t* h, const void* x, int B, int k1, int k2, void* y,
+                                            void* stream) {
+  prox_status_t s = check_common(h, x, B);
+  if (s != PROX_OK) return s;
+  if (!y || !aligned16(y)) return PROX_ERR_INVALID_ARG;
+  if (k1 < 1 || k1 > h->cfg.d_model || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  if (!h->svals) {
+    if (dev_alloc(&h->svals, (size_t)h->cfg.max_batch * F) != cudaSuccess) return PROX_ERR_OOM;
+  }
+  h->sel_unordered = 0;
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st, h->svals)) != PROX_OK) return s;
+  if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
+  {
+    LaunchScope ls(h, kKGateUp, st);
+    dim3 g((k2 + 255) / 256, B);
+    gather_values_kernel<<<g, 256, 0, st>>>(h->svals, h->sel, F, k2, F, h->hbuf, F, h->dev_status);
+  }
+  CK(cudaGetLastError());
+  return launch_down(h, B, h->sel, F, nullptr, k2, y, st);
 }
 
 prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* info) {
@@ -917,7 +974,7 @@ prox_status_t prox_algorithmic_bytes(const prox_ffn_t* h, int rows_in, int rows_
   if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
   const int64_t D = h->cfg.d_model, F = h->cfg.d_ff;
   const int64_t ngroups = D / h->group;
-  if (stage1) *stage1 = (int64_t)rows_in * F * h->bits / 4 + 2 * ngroups * F * 2;
+  if (stage1) *stage1 = (int64_t)rows_in * F * h->bits / 4 + (h->bits == 16 ? 0 : 2 * ngroups * F * 2);
   if (gate_up) *gate_up = 2 * (int64_t)rows_ch * D * 2;
   if (down) *down = (int64_t)rows_ch * D * 2;
   if (activations) *activations = 4 * D + 8 * F + 16 * (int64_t)rows_ch + (h->cfg.out_dtype ? 4 : 2) * D;
@@ -928,6 +985,7 @@ prox_status_t prox_algorithmic_bytes(const prox_ffn_t* h, int rows_in, int rows_
 prox_status_t prox_proxy_export(prox_ffn_t* h, int which, int8_t* q_host, float* scale_host) {
   if (!h || !q_host || !scale_host || (which != 0 && which != 1)) return PROX_ERR_INVALID_ARG;
   if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  if (h->bits == 16) return PROX_ERR_UNSUPPORTED;        // no integer codes to export
   CK(cudaDeviceSynchronize());
   const int D = h->cfg.d_model, F = h->cfg.d_ff, bits = h->bits;
   const int CH = ch_per_chunk(bits), nchunks = F / CH, ngroups = D / h->group;
@@ -1003,7 +1061,7 @@ prox_status_t prox_pack_load(prox_ffn_t* h, const char* path, void* stream) {
     return PROX_ERR_IO;
   }
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
-  const bool shape_ok = hd.d_model == D && hd.d_ff == F && (hd.bits == 4 || hd.bits == 8) &&
+  const bool shape_ok = hd.d_model == D && hd.d_ff == F && (hd.bits == 4 || hd.bits == 8 || hd.bits == 16) &&
                         (hd.group == D || hd.group == 128);
   if (!shape_ok) { std::fclose(f); return PROX_ERR_INVALID_ARG; }
   prox_status_t s = alloc_packed(h, hd.bits, hd.group);

@@ -186,6 +186,24 @@ __global__ void proxy_pack_kernel(const __nv_bfloat16* __restrict__ wg,
   P[(size_t)i * words_per_row + wword] = out;
 }
 
+// 16-bit "proxies" (ablation A1 of Sec. "Ablation Studies"; also the 16-bit input-sparse GEMV that
+// the cost ratio alpha of Sec. 4.2 is measured against): the original bf16 weights in the proxies'
+// input-major order.  A 16-byte chunk of row i holds 4 channels: words 0,1 gate, words 2,3 up.
+// One thread per 32-bit word (two channels of one matrix).
+__global__ void proxy_pack16_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__ wu,
+                                    int D, int F, uint32_t* __restrict__ P) {
+  const long long words_per_row = (long long)(F / 4) * 4;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid >= words_per_row * D) return;
+  const int i = (int)(tid % D);                    // consecutive threads: consecutive inputs (coalesced reads)
+  const long long wword = tid / D;
+  const int chunk = (int)(wword >> 2), word = (int)(wword & 3);
+  const uint16_t* w = (word >> 1) ? wu : wg;
+  const int j0 = chunk * 4 + (word & 1) * 2;
+  P[(size_t)i * words_per_row + wword] =
+      (uint32_t)w[(size_t)j0 * D + i] | ((uint32_t)w[(size_t)(j0 + 1) * D + i] << 16);
+}
+
 // W_down [D, F] -> channel-major [F, D]  (Sec. 3.1: y = sum_j s_j W_down[j,:]).
 __global__ void transpose_bf16_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
                                       int rows, int cols) {
@@ -296,7 +314,7 @@ input_select_kernel(const uint16_t* __restrict__ x, int D, int k1, float tau, in
 // ----------------------------------------------------------------------------
 template <int BITS>
 struct ProxyFmt {
-  static constexpr int CH = (BITS == 4) ? 16 : 8;    // channels per 16-byte chunk
+  static constexpr int CH = (BITS == 4) ? 16 : (BITS == 8 ? 8 : 4);    // channels per 16-byte chunk
   static constexpr int NACC = 2 * CH;
 };
 
@@ -314,7 +332,7 @@ __device__ __forceinline__ void proxy_accumulate(const uint4& v, float xv, float
         acc[q * 8 + m] = fmaf(f, xv, acc[q * 8 + m]);
       }
     }
-  } else {
+  } else if (BITS == 8) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
 #pragma unroll
@@ -323,6 +341,12 @@ __device__ __forceinline__ void proxy_accumulate(const uint4& v, float xv, float
         const float f = __uint_as_float(bits) - 8388736.0f;     // 2^23 + 128
         acc[q * 4 + m] = fmaf(f, xv, acc[q * 4 + m]);
       }
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {                               // bf16 weights as they are
+      acc[q * 2] = fmaf(__uint_as_float(w[q] << 16), xv, acc[q * 2]);
+      acc[q * 2 + 1] = fmaf(__uint_as_float(w[q] & 0xffff0000u), xv, acc[q * 2 + 1]);
     }
   }
 }
@@ -362,7 +386,7 @@ proxy_gemv_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
                   const uint16_t* __restrict__ x, const int* __restrict__ idx, int idx_stride,
                   const int* __restrict__ cnt, int k1_static, int D, int F, int gshift,
                   float* __restrict__ part, unsigned* __restrict__ ticket,
-                  float* __restrict__ scores, int* __restrict__ status) {
+                  float* __restrict__ scores, float* __restrict__ values, int* __restrict__ status) {
   constexpr int CH = ProxyFmt<BITS>::CH, NACC = ProxyFmt<BITS>::NACC;
   constexpr int U = 8;
   extern __shared__ float red[];                    // [warps][NACC*32]
@@ -390,9 +414,14 @@ proxy_gemv_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
 
   auto flush = [&](int g) {
     if (g < 0 || !valid) return;
+    if (BITS == 16) {                                 // no scales: the weights themselves
+#pragma unroll
+      for (int c = 0; c < NACC; ++c) { tot[c] += acc[c]; acc[c] = 0.f; }
+      return;
+    }
     const uint4* sp = reinterpret_cast<const uint4*>(S + ((size_t)g * nchunks + chunk) * NACC);
 #pragma unroll
-    for (int v4 = 0; v4 < NACC / 8; ++v4) {
+    for (int v4 = 0; v4 < (NACC >= 8 ? NACC / 8 : 1); ++v4) {
       const uint4 sv = __ldg(sp + v4);
       const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
@@ -493,7 +522,9 @@ proxy_gemv_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
     const int ch = (strip * 32 + ln) * CH + c;
     if (ch < F) {
       const float g = fin[k], u = fin[k + CH * 32];
-      scores[(size_t)b * F + ch] = fabsf(u * silu_fast(g));
+      const float v = u * silu_fast(g);
+      scores[(size_t)b * F + ch] = fabsf(v);
+      if (values) values[(size_t)b * F + ch] = v;     // signed s~, for the proxy-values-into-down variant
     }
   }
 }
@@ -626,6 +657,17 @@ gateup_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__ wu,
   ag = warp_sum(ag);
   au = warp_sum(au);
   if (lane == 0) h_out[(size_t)b * h_stride + r] = au * silu_exact(ag);
+}
+
+// Proxy values into the down projection (ablation A3): h_r = s~[sel[r]].
+__global__ void gather_values_kernel(const float* __restrict__ values, const int* __restrict__ sel,
+                                     int sel_stride, int k2, int F, float* __restrict__ h_out, int h_stride,
+                                     int* __restrict__ status) {
+  const int b = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= k2) return;
+  const int j = sel[(size_t)b * sel_stride + r];
+  if (j < 0 || j >= F) { atomicOr(status, kBadChannel); h_out[(size_t)b * h_stride + r] = 0.f; return; }
+  h_out[(size_t)b * h_stride + r] = values[(size_t)b * F + j];
 }
 
 // ----------------------------------------------------------------------------

@@ -37,6 +37,8 @@ class Problem:
         self.pb.prox_quantize_proxy(self.h, bits, group)
         torch.cuda.synchronize()
         self.fmt = (bits, group)
+        if bits == 16 and self.fmt not in self.deq:
+            self.deq[self.fmt] = (self.wg, self.wu, None)      # 16-bit proxy: the original weights
         if self.fmt not in self.deq:
             qg, sg = po.quantize_proxy(self.wg, bits, group)
             qu, su = po.quantize_proxy(self.wu, bits, group)

@@ -448,6 +448,50 @@ def test_threshold_variant(pb, toy):
 
 
 # ------------------------------------------------------------- pack save/load
+# ------------------------------------------------------------ ablation forms
+@pytest.mark.parametrize("B", [1, 3, 8])
+def test_sixteen_bit_proxy_forward(pb, toy, B):
+    """Ablation A1: the original bf16 weights, input-major, as the proxy."""
+    wl, p = toy
+    p.quantize(16, 0)
+    k1, k2 = wl.points[50]
+    for t in (0, 9):
+        _forward_check(pb, p, t, k1, k2, B=B)
+    _forward_check(pb, p, 1, p.D, 300, B=B)          # exact scores: the mask is the top-k of |s|
+    assert pb.prox_last_device_status(p.h) == 0
+    R = pb.raw
+    assert R("prox_quantize_proxy")(p.h, 16, 128, None) == 2
+    q = np.empty((p.F, p.D), dtype=np.int8)
+    s = np.empty((p.F, 1), dtype=np.float32)
+    assert R("prox_proxy_export")(p.h, 0, q.ctypes.data, s.ctypes.data) == 2
+
+
+@pytest.mark.parametrize("bits,group,B", [(4, 0, 1), (4, 128, 4), (8, 0, 2), (16, 0, 1), (16, 0, 8)])
+def test_proxy_values_into_down(pb, toy, bits, group, B):
+    """Ablation A3 (with 16-bit proxies: input sparsity on x, then on s): the selected proxy values
+    enter the down projection."""
+    wl, p = toy
+    dg, du, _ = p.quantize(bits, group)
+    for k1, k2 in (wl.points[50], (p.D, p.F), (37, 1)):
+        t = 5
+        y = p.y_empty(B)
+        used = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        pb.prox_ffn_forward_proxy_values(p.h, p.t_x[t:t + B], B, k1, k2, y)
+        pb.prox_ffn_last_mask(p.h, B, k2, used)
+        torch.cuda.synchronize()
+        used_np, y_np = used.cpu().numpy().astype(np.int64), y.float().cpu().numpy()
+        for b in range(B):
+            idx, score, sel_ref, thr = p.oracle_stage1(t + b, k1, k2)
+            check_mask(used_np[b], score, sel_ref, thr, k2, p.F)
+            vals = po.proxy_values(p.x[t + b], idx, dg, du)
+            y_ref = p.wd[:, used_np[b]].astype(np.float64) @ vals[used_np[b]]
+            check_y(y_np[b], y_ref)
+            if k1 == p.D and k2 == p.F and bits == 16:       # nothing dropped, exact proxy: the dense FFN
+                y_dense, _ = po.dense_ffn(p.x[t + b], p.wg, p.wu, p.wd)
+                check_y(y_np[b], y_dense)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
 def test_pack_save_load_roundtrip(pb, toy, tmp_path):
     wl, p = toy
     p.quantize(4, 128)
