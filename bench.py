@@ -51,6 +51,8 @@ def parse():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--alpha", action="store_true",
+                    help="also measure the proxy-cost ratio alpha (integer proxy GEMV / 16-bit GEMV at equal input sparsity)")
     return ap.parse_args()
 
 
@@ -398,6 +400,59 @@ def run_prox(args):
                   "dense_cublas_bf16_us_per_call": d8_us / calls8 if d8_us else None,
                   "masks": "per token; weights read once for the union"}
 
+        # Proxy-cost ratio alpha (appendix "Empirical Proxy-Cost Ratios"): latency of the integer proxy
+        # GEMV over that of the 16-bit GEMV at the same input sparsity, both by the step-wise kernel,
+        # every call on another weight replica (cold HBM).
+        alpha = None
+        if args.alpha and rank == 0 and world == 1:
+            sel1 = torch.empty(1, k2, dtype=torch.int32, device=dev)
+
+            def stage1_times(k1a):
+                def step():
+                    cs = torch.cuda.current_stream().cuda_stream
+                    for t in range(T):
+                        pb.prox_stage1_mask(handles[t % R], x[t], 1, k1a, k2, sel1, stream=cs)
+                whole = timed_graph(step)
+                for h in handles:
+                    pb.prox_profile_enable(h, 1)
+                for t in range(T):
+                    pb.prox_stage1_mask(handles[t % R], x[t], 1, k1a, k2, sel1, stream=sp)
+                stream.synchronize()
+                n, tot = 0, 0.0
+                for h in handles:
+                    c, m = pb.prox_profile_read(h)["proxy_gemv"]
+                    n += c; tot += m
+                    pb.prox_profile_enable(h, 0)
+                return (whole / T if whole else None), tot / max(n, 1) * 1e3
+
+            levels = (0.0, 0.10, 0.55, 0.70)
+            res = {}
+            for fmt in (PROXY, (16, 0)):
+                for h in handles:
+                    pb.prox_quantize_proxy(h, *fmt)
+                torch.cuda.synchronize()
+                base_whole, _ = stage1_times(1)                  # one input row: everything but the streaming
+                for s1 in levels:
+                    k1a = pb.prox_sparsity_to_k(s1, D)
+                    whole, kern = stage1_times(k1a)
+                    res[(fmt[0], s1)] = {"k1": k1a, "gemv_kernel_us": kern, "stage1_us": whole,
+                                         "stage1_us_one_row": base_whole}
+            for h in handles:
+                pb.prox_quantize_proxy(h, *PROXY)
+            torch.cuda.synchronize()
+            alpha = {"proxy": f"int{PROXY[0]} group-{PROXY[1]}", "against": "bf16 input-major rows, same kernel template",
+                     "levels": []}
+            for s1 in levels:
+                lo, hi = res[(PROXY[0], s1)], res[(16, s1)]
+                marg = None
+                if lo["stage1_us"] and hi["stage1_us"] and hi["stage1_us"] > hi["stage1_us_one_row"]:
+                    marg = (lo["stage1_us"] - lo["stage1_us_one_row"]) / (hi["stage1_us"] - hi["stage1_us_one_row"])
+                alpha["levels"].append({"input_sparsity": s1, "k1": lo["k1"],
+                                        "int_gemv_us": lo["gemv_kernel_us"], "bf16_gemv_us": hi["gemv_kernel_us"],
+                                        "alpha_kernel_events": lo["gemv_kernel_us"] / hi["gemv_kernel_us"],
+                                        "int_stage1_us": lo["stage1_us"], "bf16_stage1_us": hi["stage1_us"],
+                                        "alpha_marginal": marg})
+
     ms, e2e_ms = max_over_ranks([ms, e2e_s * 1e3], dev)
     us_per_call = whole_job_us_per_call(ms, world, args.steps, T)
     e2e_us = whole_job_us_per_call(e2e_ms, world, e2e_steps, T)
@@ -459,6 +514,7 @@ def run_prox(args):
             "gpu_launches": int(round(launches_per_call * T * args.steps)),
             "dense_cublas_bf16_us_per_call": dense_us,
             "batch8": batch8,
+            "alpha": alpha,
             "clocks": clocks,
         }
         print(json.dumps(out))

@@ -131,10 +131,22 @@ int nstrips_for(int F, int bits) {
   return (F + per_strip - 1) / per_strip;
 }
 
+// Row split of the step-wise proxy GEMV: as many blocks as are resident at once (one wave; a few
+// blocks more would run as a second wave and double the time).
 int ksplit_for(const prox_ffn* h, int B, int n_rows) {
   const int ns = nstrips_for(h->cfg.d_ff, h->bits);
-  int target = 2 * h->sm_count;
-  int ks = (target + ns * B - 1) / (ns * B);
+  static int occ[3] = {0, 0, 0};
+  const int fi = h->bits == 4 ? 0 : (h->bits == 8 ? 1 : 2);
+  if (!occ[fi]) {
+    int nb = 0;
+    const void* fn = fi == 0 ? (const void*)proxy_gemv_kernel<4> : fi == 1 ? (const void*)proxy_gemv_kernel<8>
+                                                                           : (const void*)proxy_gemv_kernel<16>;
+    const size_t smem = (size_t)kProxyWarps * 2 * ch_per_chunk(h->bits) * 32 * sizeof(float);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kProxyThreads, smem) != cudaSuccess || nb < 1) nb = 1;
+    occ[fi] = nb;
+  }
+  const int target = occ[fi] * h->sm_count;
+  int ks = target / (ns * B);
   const int by_rows = n_rows / 32 > 1 ? n_rows / 32 : 1;   // keep >= 4 rows per warp
   if (ks > by_rows) ks = by_rows;
   if (ks > 32) ks = 32;

@@ -381,7 +381,7 @@ __device__ __forceinline__ void proxy_accumulate_exact(const uint4& v, float xv,
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kProxyThreads)
+__global__ void __launch_bounds__(kProxyThreads, BITS == 16 ? 3 : 2)
 proxy_gemv_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S,
                   const uint16_t* __restrict__ x, const int* __restrict__ idx, int idx_stride,
                   const int* __restrict__ cnt, int k1_static, int D, int F, int gshift,
