@@ -24,7 +24,8 @@ paper; the paper's closed forms q_Lap, q_G, eta, Corr; the residual bound
 ||xW - x_sp W|| <= ||r|| ||W||; the order-preservation condition; quantizer
 invariants; a hand-worked 4x4 example; the ablation forms against the dense FFN
 (all inputs and channels kept, original weights as proxy) and against Stage 2 on
-the exact top-k of |s|.  The mask and output *values* on random
+the exact top-k of |s|; RMSNorm against the library's rms_norm and the layer
+block against its parts.  The mask and output *values* on random
 inputs have no worked example in the paper: parity unpinned for those beyond
 the properties above.
 """
@@ -37,6 +38,7 @@ __all__ = [
     "dequantize", "input_topk", "input_threshold", "input_sparse_projection", "proxy_scores", "channel_topk",
     "channel_threshold", "stage2", "forward", "forward_batch", "allocate_budget",
     "sparsity_to_k", "effective_sparsity", "proxy_values", "forward_proxy_values",
+    "rmsnorm", "ffn_block", "ffn_stack",
 ]
 
 
@@ -238,6 +240,43 @@ def forward_batch(xs, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down):
     """Tokens are independent: every token gets its own masks (the paper treats
     single-batch decoding only)."""
     return [forward(x, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down) for x in xs]
+
+
+# ------------------------------------------------ the FFN sub-block of a layer
+def rmsnorm(x, w, eps: float) -> np.ndarray:
+    """RMSNorm as the models of the paper's evaluation (Qwen3, Llama-3) define
+    it: x_i / sqrt(mean(x^2) + eps) * w_i.  The paper only names it (appendix
+    "End-to-End Latency Analysis": attention, RMSNorm and residual around the
+    FFN); this is the standard definition."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    ms = 0.0
+    for v in x:                       # plain running sum, one element after the other
+        ms += v * v
+    inv = 1.0 / np.sqrt(ms / x.shape[0] + eps)
+    return x * inv * w
+
+
+def ffn_block(x_res, norm_w, eps: float, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down):
+    """One layer's FFN sub-block on the residual stream (pre-norm decoder layer):
+        x_res' = x_res + ProxFFN(bf16(RMSNorm(x_res) * w)).
+    The FFN input is rounded to bf16, the dtype of the FFN's activations and
+    weights; the residual stream itself is kept unrounded here.  Returns
+    (x_res', dict of the FFN call, FFN input as float64)."""
+    xn = bf16_to_f64(f64_to_bf16_bits(rmsnorm(x_res, norm_w, eps)))
+    out = forward(xn, k1, k2, deq_gate, deq_up, w_gate, w_up, w_down)
+    return np.asarray(x_res, dtype=np.float64) + out["y"], out, xn
+
+
+def ffn_stack(x_res, layers, eps: float, k1: int, k2: int):
+    """`layers` = list of (norm_w, deq_gate, deq_up, w_gate, w_up, w_down): the
+    FFN sub-blocks of consecutive layers applied to one residual stream (the
+    attention sub-blocks between them are outside the method).  Returns the list
+    of residual streams [before layer 0, after layer 0, ...]."""
+    xs = [np.asarray(x_res, dtype=np.float64)]
+    for (nw, dg, du, wg, wu, wd) in layers:
+        xs.append(ffn_block(xs[-1], nw, eps, k1, k2, dg, du, wg, wu, wd)[0])
+    return xs
 
 
 # ---------------------------------------------------------- budget helper
