@@ -400,6 +400,23 @@ def run_prox(args):
                   "dense_cublas_bf16_us_per_call": d8_us / calls8 if d8_us else None,
                   "masks": "per token; weights read once for the union"}
 
+        # The FFN sub-blocks of a 36-layer decoder applied to one residual stream, one graph per token
+        # (RMSNorm + Prox FFN + residual add per layer in one launch each; layer l reads replica l mod R).
+        LAYERS = 36
+        nw = (1.0 + 0.1 * torch.randn(LAYERS, D, generator=gen, device=dev, dtype=torch.float32)).to(torch.bfloat16)
+        xr0 = x[:1].float().contiguous()
+        xr = xr0.clone()
+        stack_handles = [handles[l % R] for l in range(LAYERS)]
+
+        def stack_step():
+            xr.copy_(xr0)
+            pb.prox_ffn_stack_forward(stack_handles, nw, 1e-6, xr, 1, k1, k2, None,
+                                      stream=torch.cuda.current_stream().cuda_stream)
+        stack_us = timed_graph(stack_step, reps=10)
+        decode_stack = {"layers": LAYERS, "ms_per_token": stack_us / 1e3 if stack_us else None,
+                        "us_per_layer": stack_us / LAYERS if stack_us else None,
+                        "what": "RMSNorm + Prox FFN + residual per layer, fp32 residual stream, batch 1"}
+
         # Proxy-cost ratio alpha (appendix "Empirical Proxy-Cost Ratios"): latency of the integer proxy
         # GEMV over that of the 16-bit GEMV at the same input sparsity, both by the step-wise kernel,
         # every call on another weight replica (cold HBM).
@@ -514,6 +531,7 @@ def run_prox(args):
             "gpu_launches": int(round(launches_per_call * T * args.steps)),
             "dense_cublas_bf16_us_per_call": dense_us,
             "batch8": batch8,
+            "decode_stack": decode_stack,
             "alpha": alpha,
             "clocks": clocks,
         }

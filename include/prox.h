@@ -236,6 +236,34 @@ prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x_dev, int B
 prox_status_t prox_ffn_forward_proxy_values(prox_ffn_t* h, const void* x_dev, int B, int k1, int k2,
                                             void* y_dev, void* stream);
 
+/* One layer's FFN sub-block on the residual stream (pre-norm decoder layer; the
+ * appendix "End-to-End Latency Analysis" counts RMSNorm and the residual around
+ * the FFN into the per-token time of a layer):
+ *     x_res' = x_res + ProxFFN( bf16( x_res / sqrt(mean(x_res^2) + eps) * norm_w ) ).
+ *   x_res      dev fp32 [B, d_model]  the residual stream (read)
+ *   norm_w     dev bf16 [d_model]     RMSNorm weight
+ *   x_res_out  dev fp32 [B, d_model]  result; may be x_res itself (in place)
+ * The norm is evaluated in fp64 and rounded once to bf16, so that the FFN input,
+ * on which both masks depend, is the nearest bf16 of the exact value.  At B = 1
+ * norm, FFN and residual add are one launch of the persistent kernel; otherwise
+ * one small norm kernel precedes the batch path and its last kernel adds x_res.
+ * The handle's out_dtype is not used.  Errors as prox_ffn_forward. */
+prox_status_t prox_ffn_block_forward(prox_ffn_t* h, const float* x_res_dev, const void* norm_w_dev,
+                                     double eps, int B, int k1, int k2, float* x_res_out_dev, void* stream);
+
+/* The FFN sub-blocks of n_layers consecutive layers applied in place to one
+ * residual stream (the attention sub-blocks between them are outside the
+ * method): one prox_ffn_block_forward per layer, enqueued back to back.
+ *   layers     host array of n_layers handles (same d_model)
+ *   norm_w     dev bf16 [n_layers, d_model]
+ *   x_res      dev fp32 [B, d_model], in and out
+ *   trace      NULL, or dev fp32 [n_layers + 1, B, d_model]: the stream before
+ *              layer 0 and after every layer (for checking a stack layer by layer)
+ * Errors: INVALID_ARG, and those of prox_ffn_block_forward. */
+prox_status_t prox_ffn_stack_forward(prox_ffn_t* const* layers, int n_layers, const void* norm_w_dev,
+                                     double eps, float* x_res_dev, int B, int k1, int k2,
+                                     float* trace_dev_or_null, void* stream);
+
 /* Runtime mask counts accumulated by the threshold entry points since the last
  * reset (appendix "Threshold Calibration and Runtime Sparsity":
  * e^ = s2^ - 2 alpha (1 - s1^) / 3).  Host-synchronous.  Any pointer may be NULL. */

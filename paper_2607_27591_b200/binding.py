@@ -53,6 +53,8 @@ _SIGS = {
     "prox_stage2_ffn_var": [_vp, _vp, _i, _vp, _vp, _vp, _vp],
     "prox_ffn_forward_threshold": [_vp, _vp, _i, _f, _f, _vp, _vp],
     "prox_ffn_forward_proxy_values": [_vp, _vp, _i, _i, _i, _vp, _vp],
+    "prox_ffn_block_forward": [_vp, _vp, _vp, _d, _i, _i, _i, _vp, _vp],
+    "prox_ffn_stack_forward": [C.POINTER(_vp), _i, _vp, _d, _vp, _i, _i, _i, _vp, _vp],
     "prox_runtime_sparsity": [_vp, _d, C.POINTER(C.c_int64), C.POINTER(_d), C.POINTER(_d), C.POINTER(_d), _i],
     "prox_allocate_budget": [_d, _d, _d, _d, _d, C.POINTER(_d), C.POINTER(_d)],
     "prox_sparsity_to_k": [_d, _i, C.POINTER(_i)],
@@ -201,6 +203,19 @@ def prox_ffn_forward_threshold(handle: int, x, B: int, tau_x: float, tau_s: floa
 def prox_ffn_forward_proxy_values(handle: int, x, B: int, k1: int, k2: int, y, stream=None) -> None:
     _check(_lib.prox_ffn_forward_proxy_values(handle, _ptr(x), B, k1, k2, _ptr(y), _ptr(stream)),
            "prox_ffn_forward_proxy_values")
+
+
+def prox_ffn_block_forward(handle: int, x_res, norm_w, eps: float, B: int, k1: int, k2: int, x_res_out,
+                           stream=None) -> None:
+    _check(_lib.prox_ffn_block_forward(handle, _ptr(x_res), _ptr(norm_w), eps, B, k1, k2, _ptr(x_res_out),
+                                       _ptr(stream)), "prox_ffn_block_forward")
+
+
+def prox_ffn_stack_forward(handles, norm_w, eps: float, x_res, B: int, k1: int, k2: int, trace=None,
+                           stream=None) -> None:
+    arr = (_vp * len(handles))(*handles)
+    _check(_lib.prox_ffn_stack_forward(arr, len(handles), _ptr(norm_w), eps, _ptr(x_res), B, k1, k2,
+                                       _ptr(trace), _ptr(stream)), "prox_ffn_stack_forward")
 
 
 def prox_runtime_sparsity(handle: int, alpha: float = 1.0 / 3.0, reset: bool = False):

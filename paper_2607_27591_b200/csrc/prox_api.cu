@@ -42,6 +42,9 @@ struct prox_ffn {
   unsigned* ticket;         // [maxB][nstrips_max]
   float* scores;            // [maxB][F]
   float* svals;             // [maxB][F] signed proxy values (proxy-values-into-down variant), on first use
+  uint16_t* xn;             // [maxB][D] bf16 FFN input of the layer sub-block form (step-wise path), on first use
+  const float* fin_resid;   // while a layer sub-block call is enqueued: the residual stream to add ...
+  float* fin_out;           // ... and where the sum goes
   int* sel;                 // [maxB][F]
   int* cnt_s;               // [maxB]
   float* hbuf;              // [maxB][F]
@@ -263,7 +266,8 @@ prox_status_t launch_down(prox_ffn* h, int B, const int* sel, int stride, const 
   const int n = B * D;
   {
     LaunchScope ls(h, kKFinalize, st);
-    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, y, n, h->cfg.out_dtype);
+    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, h->fin_resid ? (void*)h->fin_out : y, n,
+                                                     h->cfg.out_dtype, h->fin_resid);
   }
   CK(cudaGetLastError());
   return PROX_OK;
@@ -457,7 +461,8 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   const int n = B * D;
   {
     LaunchScope ls(h, kKFinalize, st);
-    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, y, n, h->cfg.out_dtype);
+    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, h->fin_resid ? (void*)h->fin_out : y, n,
+                                                     h->cfg.out_dtype, h->fin_resid);
   }
   CK(cudaGetLastError());
   return PROX_OK;
@@ -507,10 +512,10 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   return pl;
 }
 
-template <int BITS, int NG>
-cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
+template <int BITS, int NG, bool NORM>
+cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
   static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
-  auto kern = prox_fused_kernel<BITS, NG>;
+  auto kern = prox_fused_kernel<BITS, NG, NORM>;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
@@ -530,8 +535,23 @@ cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStre
   return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
+template <int BITS, int NG>
+cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
+  return prm.xres ? launch_fused_tn<BITS, NG, true>(pl, prm, st) : launch_fused_tn<BITS, NG, false>(pl, prm, st);
+}
+
+// 1/d_model and eps as pairs of floats for the device-side RMSNorm
+RmsConst rms_const(int D, double eps) {
+  RmsConst c;
+  const double inv_d = 1.0 / (double)D;
+  c.idh = (float)inv_d; c.idl = (float)(inv_d - (double)c.idh);
+  c.eh = (float)eps; c.el = (float)(eps - (double)c.eh);
+  return c;
+}
+
 prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int k1, int k2, void* y,
-                           int* sel_out, cudaStream_t st) {
+                           int* sel_out, cudaStream_t st, const float* xres = nullptr,
+                           const uint16_t* norm_w = nullptr, double eps = 0.0, float* xres_out = nullptr) {
   FusedParams prm;
   std::memset(&prm, 0, sizeof(prm));
   prm.P = h->P; prm.S = h->S; prm.wg = h->wg; prm.wu = h->wu; prm.wdt = h->wdt;
@@ -546,6 +566,7 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.status = h->dev_status;
   prm.big_bytes = pl.big_bytes; prm.nslots = pl.nslots;
   prm.trace = h->trace;
+  prm.xres = xres; prm.norm_w = norm_w; prm.rc = rms_const(h->cfg.d_model, eps); prm.xres_out = xres_out;
   cudaError_t e;
   {
     LaunchScope ls(h, kKFused, st);
@@ -559,6 +580,22 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   }
   CK(e);
   return PROX_OK;
+}
+
+// Everything of a forward call but the persistent kernel: batch path, or the step-wise kernels.
+prox_status_t forward_kernels(prox_ffn* h, const void* x, int B, int k1, int k2, void* y, cudaStream_t st) {
+  prox_status_t s;
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  h->sel_unordered = 0;
+  if (h->use_union && batch_path_ok(h, B, true)) {
+    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
+    return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
+  }
+  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
+  if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
+  if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
+  if (h->use_union && batch_path_ok(h, B)) return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, false);
+  return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
 }
 
 }  // namespace
@@ -651,7 +688,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   if (!h) return;
   free_packed(h);
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
-  cudaFree(h->scores); cudaFree(h->svals); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
+  cudaFree(h->scores); cudaFree(h->svals); cudaFree(h->xn); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
   cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->cmask); cudaFree(h->umask);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
@@ -760,16 +797,59 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x, int B, int k1, int 
     const FusedPlan pl = plan_fused(h, k1, k2);
     if (pl.ok) { h->sel_unordered = 1; return launch_fused(h, pl, x, k1, k2, y, h->sel, st); }
   }
-  h->sel_unordered = 0;
-  if (h->use_union && batch_path_ok(h, B, true)) {
-    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
-    return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
+  return forward_kernels(h, x, B, k1, k2, y, st);
+}
+
+/* One layer's FFN sub-block on the residual stream. */
+prox_status_t prox_ffn_block_forward(prox_ffn_t* h, const float* x_res, const void* norm_w, double eps, int B,
+                                     int k1, int k2, float* x_res_out, void* stream) {
+  prox_status_t s = check_common(h, x_res, B);
+  if (s != PROX_OK) return s;
+  if (!norm_w || !x_res_out || !aligned16(x_res_out) || !aligned16(norm_w)) return PROX_ERR_INVALID_ARG;
+  if (!(eps >= 0.0)) return PROX_ERR_INVALID_ARG;
+  if (k1 < 1 || k1 > h->cfg.d_model || k2 < 1 || k2 > h->cfg.d_ff) return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model;
+  if (B == 1) {
+    const FusedPlan pl = plan_fused(h, k1, k2);
+    if (pl.ok) {
+      h->sel_unordered = 1;
+      return launch_fused(h, pl, nullptr, k1, k2, nullptr, h->sel, st, x_res,
+                          static_cast<const uint16_t*>(norm_w), eps, x_res_out);
+    }
   }
-  if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
-  if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st)) != PROX_OK) return s;
-  if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
-  if (h->use_union && batch_path_ok(h, B)) return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, false);
-  return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
+  if (!h->xn) {
+    if (dev_alloc(&h->xn, (size_t)h->cfg.max_batch * D) != cudaSuccess) return PROX_ERR_OOM;
+  }
+  rmsnorm_kernel<<<B, 256, 0, st>>>(x_res, static_cast<const uint16_t*>(norm_w), rms_const(D, eps), D, h->xn);
+  h->launches++;
+  CK(cudaGetLastError());
+  h->fin_resid = x_res; h->fin_out = x_res_out;          // the last kernel adds the residual stream
+  s = forward_kernels(h, h->xn, B, k1, k2, nullptr, st);
+  h->fin_resid = nullptr; h->fin_out = nullptr;
+  return s;
+}
+
+/* The FFN sub-blocks of consecutive layers applied to one residual stream. */
+prox_status_t prox_ffn_stack_forward(prox_ffn_t* const* layers, int n_layers, const void* norm_w, double eps,
+                                     float* x_res, int B, int k1, int k2, float* trace, void* stream) {
+  if (!layers || n_layers < 1 || !norm_w || !x_res) return PROX_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!layers[l]) return PROX_ERR_INVALID_ARG;
+    if (layers[l]->cfg.d_model != layers[0]->cfg.d_model) return PROX_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t D = (size_t)layers[0]->cfg.d_model;
+  const size_t bytes = (size_t)B * D * sizeof(float);
+  if (trace) CK(cudaMemcpyAsync(trace, x_res, bytes, cudaMemcpyDeviceToDevice, st));
+  for (int l = 0; l < n_layers; ++l) {
+    const prox_status_t s = prox_ffn_block_forward(layers[l], x_res, static_cast<const uint16_t*>(norm_w) + (size_t)l * D,
+                                                   eps, B, k1, k2, x_res, stream);
+    if (s != PROX_OK) return s;
+    if (trace) CK(cudaMemcpyAsync(trace + (size_t)(l + 1) * B * D, x_res, bytes, cudaMemcpyDeviceToDevice, st));
+  }
+  return PROX_OK;
 }
 
 // Ablation A3 of Sec. "Ablation Studies": Stage 1 as always, then the selected proxy values themselves

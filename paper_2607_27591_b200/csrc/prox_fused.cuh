@@ -59,6 +59,9 @@ struct FusedParams {
   int big_bytes;      // bytes of the large shared buffer
   int nslots;         // ring slots of D*2 bytes inside it
   unsigned long long* trace;   // optional [grid][32] phase time stamps (ns), NULL = off
+  // Layer sub-block form (all NULL / 0 otherwise): the input is bf16(RMSNorm(xres) * norm_w) and the
+  // result is xres + y, written as fp32 to xres_out (which may be xres itself).
+  const float* xres; const uint16_t* norm_w; float* xres_out; RmsConst rc;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -258,10 +261,14 @@ struct FusedSmem {
   int keys_s0, keys_s1;    // ring slots [s0, s1) that overlap the keys
   int list_s0, list_s1;    // ... and the list
   unsigned slot_use[kMaxSlots];   // uses of each ring slot whose data has been seen complete
+  float nsum[kFusedWarps][2];     // RMSNorm: the warps' sums of squares (hi, lo)
+  float ninv[2];                  // ... and 1 / sqrt(mean + eps) (hi, lo)
 };
 
 // NG = warp groups of the down projection (4: d_model <= 4096, 2: <= 8192, 1: <= 16384)
-template <int BITS, int NG>
+// NORM = layer sub-block form (RMSNorm in the prologue, residual add at the end): an instantiation of its
+// own, so that the plain call carries none of its code or registers.
+template <int BITS, int NG, bool NORM = false>
 __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const FusedParams p) {
   constexpr int CH = ProxyFmt<BITS>::CH, NACC = ProxyFmt<BITS>::NACC;
   constexpr int NT = kFusedThreads;
@@ -287,7 +294,53 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   }
   if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
   if (tid < kMaxSlots) sm.slot_use[tid] = 0;
-  {
+  if (NORM) {
+    // FFN input = bf16(RMSNorm(residual stream) * norm weight), the correctly rounded value (the masks
+    // depend on it).  Every block does all of it; x and w pass through shared memory once.
+    float hi = 0.f, lo = 0.f;
+    {
+      // both loads of a round are issued before the first use (a load per dependent iteration would put
+      // the latency of global memory on every one of them)
+      const float4* x4 = reinterpret_cast<const float4*>(p.xres);
+      const uint2* w2 = reinterpret_cast<const uint2*>(p.norm_w);
+      const int n4 = D / 4;
+#pragma unroll 1
+      for (int i0 = tid; i0 < n4; i0 += 2 * NT) {
+        const int i1 = i0 + NT;
+        const bool two = i1 < n4;
+        const float4 a = __ldcg(x4 + i0);
+        const uint2 wa = __ldg(w2 + i0);
+        const float4 b = two ? __ldcg(x4 + i1) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const uint2 wb = two ? __ldg(w2 + i1) : make_uint2(0u, 0u);
+        reinterpret_cast<float4*>(xf)[i0] = a;
+        reinterpret_cast<uint2*>(idx16)[i0] = wa;
+        f2_add_square(hi, lo, a.x); f2_add_square(hi, lo, a.y); f2_add_square(hi, lo, a.z); f2_add_square(hi, lo, a.w);
+        if (two) {
+          reinterpret_cast<float4*>(xf)[i1] = b;
+          reinterpret_cast<uint2*>(idx16)[i1] = wb;
+          f2_add_square(hi, lo, b.x); f2_add_square(hi, lo, b.y); f2_add_square(hi, lo, b.z); f2_add_square(hi, lo, b.w);
+        }
+      }
+    }
+    for (int i = tid; i < 1024 + 32; i += NT) { if (i < 1024) sm.hist[i] = 0; else sm.hist2[i - 1024] = 0; }
+    f2_warp_sum(hi, lo);
+    if (lane == 0) { sm.nsum[warp][0] = hi; sm.nsum[warp][1] = lo; }
+    __syncthreads();
+    if (warp == 0) {
+      hi = lane < kFusedWarps ? sm.nsum[lane][0] : 0.f;
+      lo = lane < kFusedWarps ? sm.nsum[lane][1] : 0.f;
+      f2_warp_sum(hi, lo);
+      if (lane == 0) rms_inverse(hi, lo, p.rc, sm.ninv[0], sm.ninv[1]);
+    }
+    __syncthreads();
+    const float ih = sm.ninv[0], il = sm.ninv[1];
+#pragma unroll 1
+    for (int i = tid; i < D; i += NT) {
+      const uint16_t b = rms_scale_to_bf16(xf[i], __uint_as_float((uint32_t)idx16[i] << 16), ih, il);
+      xs[i] = b;
+      xf[i] = __uint_as_float((uint32_t)b << 16);
+    }
+  } else {
     const uint4* xg = reinterpret_cast<const uint4*>(p.x);
     for (int i = tid; i < D / 8; i += NT) {
       const uint4 v = __ldg(xg + i);
@@ -1148,18 +1201,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   __syncthreads();
   if (sm.s_last) {
     for (int i0 = tid * 4; i0 < D; i0 += NT * 4 * 4) {        // loads first: they must not queue behind the stores
-      float4 v[4];
+      float4 v[4], r[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int i = i0 + u * NT * 4;
         v[u] = (i < D) ? __ldcg(reinterpret_cast<const float4*>(p.yacc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        r[u] = (NORM && i < D) ? __ldcg(reinterpret_cast<const float4*>(p.xres + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int i = i0 + u * NT * 4;
         if (i < D) {
           *reinterpret_cast<float4*>(p.yacc + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (p.out_fp32) {
+          if (NORM) {
+            *reinterpret_cast<float4*>(p.xres_out + i) =
+                make_float4(r[u].x + v[u].x, r[u].y + v[u].y, r[u].z + v[u].z, r[u].w + v[u].w);
+          } else if (p.out_fp32) {
             *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + i) = v[u];
           } else {
             __nv_bfloat162 lo = __floats2bfloat162_rn(v[u].x, v[u].y), hi = __floats2bfloat162_rn(v[u].z, v[u].w);

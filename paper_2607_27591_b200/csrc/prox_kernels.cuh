@@ -733,13 +733,113 @@ down_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, int h
 }
 
 // Round the fp32 accumulator once to the output type and clear it for the next call.
-__global__ void finalize_kernel(float* __restrict__ yacc, void* __restrict__ y, int n, int out_fp32) {
+// With `resid` (layer sub-block form): y = resid + accumulator, fp32 (y may be resid itself).
+__global__ void finalize_kernel(float* __restrict__ yacc, void* y, int n, int out_fp32,
+                                const float* resid = nullptr) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const float v = yacc[i];
   yacc[i] = 0.f;
-  if (out_fp32) reinterpret_cast<float*>(y)[i] = v;
+  if (resid) reinterpret_cast<float*>(y)[i] = resid[i] + v;
+  else if (out_fp32) reinterpret_cast<float*>(y)[i] = v;
   else reinterpret_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
+}
+
+// ----------------------------------------------------------------------------
+// FFN input of a layer sub-block: bf16(x / sqrt(mean(x^2) + eps) * w).
+// The masks depend on this rounding, so it must be the rounding of the exact
+// value.  fp64 vector arithmetic is slow on this GPU (five fp64 operations per
+// element made the prologue of the persistent kernel 5 us longer), so the
+// element-wise work is done on pairs of floats (an unevaluated sum hi + lo, about
+// 2^-44 relative); fp64 is used for one scalar only: 1 / sqrt(mean + eps).
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ void two_sum(float a, float b, float& s, float& e) {   // a + b = s + e exactly
+  s = __fadd_rn(a, b);
+  const float bb = __fsub_rn(s, a);
+  e = __fadd_rn(__fsub_rn(a, __fsub_rn(s, bb)), __fsub_rn(b, bb));
+}
+
+// (hi, lo) += x * x
+__device__ __forceinline__ void f2_add_square(float& hi, float& lo, float x) {
+  const float p = __fmul_rn(x, x), pe = __fmaf_rn(x, x, -p);
+  float s, e;
+  two_sum(hi, p, s, e);
+  lo = __fadd_rn(lo, __fadd_rn(e, pe));
+  hi = s;
+}
+
+__device__ __forceinline__ void f2_warp_sum(float& hi, float& lo) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float oh = __shfl_xor_sync(0xffffffffu, hi, o), ol = __shfl_xor_sync(0xffffffffu, lo, o);
+    float s, e;
+    two_sum(hi, oh, s, e);
+    lo = __fadd_rn(__fadd_rn(lo, ol), e);
+    hi = s;
+  }
+}
+
+// The scalars 1/D and eps as pairs of floats, split on the host.
+struct RmsConst { float idh, idl, eh, el; };
+
+// sum of squares (hi + lo) -> 1 / sqrt(sum / D + eps) as a pair of floats, without fp64 (a chain of
+// fp64 divide and square root alone took microseconds here): pair product, pair sum, then one
+// Newton step on rsqrtf whose residual 1 - m y0^2 is formed exactly enough (about 2^-44 in the end).
+__device__ __forceinline__ void rms_inverse(float hi, float lo, const RmsConst& c, float& ih, float& il) {
+  const float ph = __fmul_rn(hi, c.idh), pe = __fmaf_rn(hi, c.idh, -ph);
+  const float pl = __fmaf_rn(lo, c.idh, __fmaf_rn(hi, c.idl, pe));
+  float s, e;
+  two_sum(ph, c.eh, s, e);
+  const float l = __fadd_rn(__fadd_rn(e, pl), c.el);
+  float mh, ml;
+  two_sum(s, l, mh, ml);                                                    // m = mean + eps
+  const float y0 = rsqrtf(mh);
+  const float a = __fmul_rn(y0, y0), ae = __fmaf_rn(y0, y0, -a);            // y0^2 = a + ae
+  const float th = __fmul_rn(mh, a), te = __fmaf_rn(mh, a, -th);            // mh a = th + te
+  const float rest = __fadd_rn(te, __fmaf_rn(mh, ae, __fmul_rn(ml, a)));
+  const float rho = __fsub_rn(__fsub_rn(1.0f, th), rest);                   // 1 - m y0^2 (1 - th is exact)
+  const float corr = __fmul_rn(__fmul_rn(0.5f, y0), rho);
+  two_sum(y0, corr, ih, il);
+}
+
+// nearest bf16 (ties to even) of x * w * (ih + il)
+__device__ __forceinline__ uint16_t rms_scale_to_bf16(float x, float w, float ih, float il) {
+  const float p = __fmul_rn(x, w), e = __fmaf_rn(x, w, -p);                 // x w = p + e exactly
+  const float q = __fmul_rn(p, ih), qe = __fmaf_rn(p, ih, -q);              // p ih = q + qe exactly
+  const float r = __fmaf_rn(p, il, __fmaf_rn(e, ih, qe));                   // the rest, to ~2^-44
+  float s, t;
+  two_sum(q, r, s, t);                                                      // s = nearest float, t = what is left
+  uint32_t u = __float_as_uint(s);
+  if ((u & 0xffffu) == 0x8000u && t != 0.f) {
+    // s sits exactly between two bf16 values: the remainder decides (towards larger magnitude or not)
+    const bool up = (t > 0.f) == (s > 0.f);
+    return (uint16_t)((u >> 16) + (up ? 1u : 0u));
+  }
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+// One block per token (the batch and step-wise paths; the persistent kernel has this in its prologue).
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ xres, const uint16_t* __restrict__ w,
+                                                      RmsConst rc, int D, uint16_t* __restrict__ out) {
+  __shared__ float wh[8], wl[8], inv[2];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* x = xres + (size_t)b * D;
+  float hi = 0.f, lo = 0.f;
+  for (int i = tid; i < D; i += 256) f2_add_square(hi, lo, x[i]);
+  f2_warp_sum(hi, lo);
+  if (lane == 0) { wh[warp] = hi; wl[warp] = lo; }
+  __syncthreads();
+  if (warp == 0) {
+    hi = lane < 8 ? wh[lane] : 0.f;
+    lo = lane < 8 ? wl[lane] : 0.f;
+    f2_warp_sum(hi, lo);
+    if (lane == 0) rms_inverse(hi, lo, rc, inv[0], inv[1]);
+  }
+  __syncthreads();
+  const float ih = inv[0], il = inv[1];
+  for (int i = tid; i < D; i += 256)
+    out[(size_t)b * D + i] = rms_scale_to_bf16(x[i], __uint_as_float((uint32_t)w[i] << 16), ih, il);
 }
 
 }  // namespace prox

@@ -492,6 +492,99 @@ def test_proxy_values_into_down(pb, toy, bits, group, B):
     assert pb.prox_last_device_status(p.h) == 0
 
 
+# ------------------------------------------------------- layer sub-block, stacks
+def _norm_weight(D, seed):
+    rng = np.random.default_rng(seed)
+    return inputs.f32_to_bf16_bits((1.0 + 0.1 * rng.standard_normal(D)).astype(np.float32))
+
+
+def _check_block(p, dg, du, x_in, nw64, eps, k1, k2, x_out, used):
+    """One token of one layer: GPU result x_out against the oracle fed with the same residual stream."""
+    xn = po.bf16_to_f64(po.f64_to_bf16_bits(po.rmsnorm(x_in, nw64, eps)))
+    idx = po.input_topk(xn, k1)
+    score = po.proxy_scores(xn, idx, dg, du)
+    sel_ref, thr = po.channel_topk(score, k2)
+    check_mask(used, score, sel_ref, thr, k2, p.F)
+    y_ref, _ = po.stage2(xn, used, p.wg, p.wu, p.wd)
+    # x_out = fp32(x_in + y): the add rounds once more, to fp32
+    check_y(x_out.astype(np.float64) - x_in, y_ref, extra_abs=float(np.max(np.abs(x_out))) * 2.0 ** -23)
+
+
+@pytest.mark.parametrize("bits,group,B", [(4, 128, 1), (4, 0, 1), (8, 0, 1), (4, 128, 3), (8, 128, 8), (16, 0, 1)])
+def test_ffn_block_forward(pb, toy, bits, group, B):
+    wl, p = toy
+    dg, du, _ = p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    eps = 1e-6
+    nw_bits = _norm_weight(p.D, 4)
+    nw64 = po.bf16_to_f64(nw_bits)
+    from tests.gpu_common import dev_bf16
+    t_nw = dev_bf16(nw_bits)
+    rng = np.random.default_rng(8)
+    x_res = (p.x[2:2 + B] * 3.7 + rng.standard_normal((B, p.D))).astype(np.float32)
+    t_x = torch.from_numpy(x_res).cuda()
+    out = torch.empty_like(t_x)
+    used = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+    pb.prox_ffn_block_forward(p.h, t_x, t_nw, eps, B, k1, k2, out)
+    pb.prox_ffn_last_mask(p.h, B, k2, used)
+    inplace = t_x.clone()
+    pb.prox_ffn_block_forward(p.h, inplace, t_nw, eps, B, k1, k2, inplace)
+    torch.cuda.synchronize()
+    assert torch.equal(t_x.cpu(), torch.from_numpy(x_res)), "the input stream was written"
+    out_np, used_np = out.cpu().numpy(), used.cpu().numpy().astype(np.int64)
+    for b in range(B):
+        _check_block(p, dg, du, x_res[b].astype(np.float64), nw64, eps, k1, k2, out_np[b], used_np[b])
+    np.testing.assert_allclose(inplace.cpu().numpy(), out_np, rtol=1e-5, atol=1e-5)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("B", [1, 2])
+def test_ffn_stack_forward_layer_by_layer(pb, B):
+    """Three layers in place on one stream; every layer is checked against the oracle on the stream the
+    GPU itself fed into it (the trace), so a mask difference inside the band in one layer does not
+    make the next one incomparable."""
+    from tests.gpu_common import dev_bf16
+    L, D, F = 3, 512, 1536
+    probs = []
+    try:
+        for l in range(L):
+            wg, wu, wd, x = inputs.make_small(D, F, 4, seed=40 + l)
+            probs.append(Problem(pb, wg, wu, wd, x, max_batch=2))
+        deqs = [q.quantize(4, 128) for q in probs]
+        nw_bits = np.stack([_norm_weight(D, 50 + l) for l in range(L)])
+        t_nw = dev_bf16(nw_bits)
+        k1, k2, eps = 154, 358, 1e-6
+        x0 = (probs[0].x[:B] * 2.0).astype(np.float32)
+        t_x = torch.from_numpy(x0).cuda()
+        trace = torch.zeros(L + 1, B, D, dtype=torch.float32, device="cuda")
+        pb.prox_ffn_stack_forward([q.h for q in probs], t_nw, eps, t_x, B, k1, k2, trace)
+        torch.cuda.synchronize()
+        tr = trace.cpu().numpy()
+        assert np.array_equal(tr[0], x0) and np.array_equal(tr[L], t_x.cpu().numpy())
+        # layer by layer, with the mask each layer used (asked for by re-running the layer on its input)
+        for l in range(L):
+            out = torch.empty(B, D, dtype=torch.float32, device="cuda")
+            used = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+            pb.prox_ffn_block_forward(probs[l].h, trace[l], t_nw[l], eps, B, k1, k2, out)
+            pb.prox_ffn_last_mask(probs[l].h, B, k2, used)
+            torch.cuda.synchronize()
+            np.testing.assert_allclose(out.cpu().numpy(), tr[l + 1], rtol=1e-5, atol=1e-5)
+            dg, du, _ = deqs[l]
+            for b in range(B):
+                _check_block(probs[l], dg, du, tr[l, b].astype(np.float64), po.bf16_to_f64(nw_bits[l]), eps, k1, k2,
+                             tr[l + 1, b], used.cpu().numpy()[b].astype(np.int64))
+        # and the oracle's own stack from the same start stays close while no mask differs
+        layers = [(po.bf16_to_f64(nw_bits[l]), deqs[l][0], deqs[l][1], probs[l].wg, probs[l].wu, probs[l].wd)
+                  for l in range(L)]
+        xs = po.ffn_stack(x0[0].astype(np.float64), layers, eps, k1, k2)
+        assert np.sqrt(np.mean((xs[L] - tr[L, 0]) ** 2)) <= 0.05 * np.sqrt(np.mean((xs[L] - xs[0]) ** 2)) + 1e-6
+        for q in probs:
+            assert pb.prox_last_device_status(q.h) == 0
+    finally:
+        for q in probs:
+            q.close()
+
+
 def test_pack_save_load_roundtrip(pb, toy, tmp_path):
     wl, p = toy
     p.quantize(4, 128)
