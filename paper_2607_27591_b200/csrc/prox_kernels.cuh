@@ -748,10 +748,10 @@ __global__ void finalize_kernel(float* __restrict__ yacc, void* y, int n, int ou
 // ----------------------------------------------------------------------------
 // FFN input of a layer sub-block: bf16(x / sqrt(mean(x^2) + eps) * w).
 // The masks depend on this rounding, so it must be the rounding of the exact
-// value.  fp64 vector arithmetic is slow on this GPU (five fp64 operations per
-// element made the prologue of the persistent kernel 5 us longer), so the
-// element-wise work is done on pairs of floats (an unevaluated sum hi + lo, about
-// 2^-44 relative); fp64 is used for one scalar only: 1 / sqrt(mean + eps).
+// value.  The arithmetic is done on pairs of floats (an unevaluated sum hi + lo,
+// about 2^-44 relative) rather than in fp64: the same result for this purpose, no
+// fp64 divide / square-root subroutines in the prologue of the persistent kernel,
+// and full-rate instructions only.
 // ----------------------------------------------------------------------------
 __device__ __forceinline__ void two_sum(float a, float b, float& s, float& e) {   // a + b = s + e exactly
   s = __fadd_rn(a, b);
@@ -782,9 +782,9 @@ __device__ __forceinline__ void f2_warp_sum(float& hi, float& lo) {
 // The scalars 1/D and eps as pairs of floats, split on the host.
 struct RmsConst { float idh, idl, eh, el; };
 
-// sum of squares (hi + lo) -> 1 / sqrt(sum / D + eps) as a pair of floats, without fp64 (a chain of
-// fp64 divide and square root alone took microseconds here): pair product, pair sum, then one
-// Newton step on rsqrtf whose residual 1 - m y0^2 is formed exactly enough (about 2^-44 in the end).
+// sum of squares (hi + lo) -> 1 / sqrt(sum / D + eps) as a pair of floats: pair product, pair sum,
+// then one Newton step on rsqrtf whose residual 1 - m y0^2 is formed exactly enough (about 2^-44
+// in the end).
 __device__ __forceinline__ void rms_inverse(float hi, float lo, const RmsConst& c, float& ih, float& il) {
   const float ph = __fmul_rn(hi, c.idh), pe = __fmaf_rn(hi, c.idh, -ph);
   const float pl = __fmaf_rn(lo, c.idh, __fmaf_rn(hi, c.idl, pe));
