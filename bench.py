@@ -417,6 +417,43 @@ def run_prox(args):
                         "us_per_layer": stack_us / LAYERS if stack_us else None,
                         "what": "RMSNorm + Prox FFN + residual per layer, fp32 residual stream, batch 1"}
 
+        # Threshold form of the masks (the paper's run-time rule, Sec. 4.1; appendix "Threshold Calibration
+        # and Runtime Sparsity"): per-layer thresholds calibrated as empirical quantiles on the first tokens
+        # of the synthetic stream (tau_x pooled over |x| at level s1; tau_s per weight replica over its
+        # proxy scores at level s2), then the same step as the headline, one launch per call.
+        threshold_mode = None
+        try:
+            s1_t, s2_t = 1.0 - k1 / D, 1.0 - k2 / F
+            ncal = 64
+            tau_x = float(torch.quantile(x[:ncal].float().abs().flatten(), s1_t))
+            sc = torch.empty(ncal, F, dtype=torch.float32, device=dev)
+            selc = torch.empty(1, F, dtype=torch.int32, device=dev)
+            cntc = torch.empty(1, dtype=torch.int32, device=dev)
+            tau_s = []
+            for r in range(R):
+                for i in range(ncal):
+                    pb.prox_stage1_mask_threshold(handles[r], x[i], 1, tau_x, 0.0, selc, cntc, sc[i], stream=sp)
+                stream.synchronize()
+                tau_s.append(float(torch.quantile(sc.flatten(), s2_t)))
+            for h in handles:
+                pb.prox_runtime_sparsity(h, reset=True)
+
+            def thr_step():
+                cs = torch.cuda.current_stream().cuda_stream
+                for t in range(T):
+                    pb.prox_ffn_forward_threshold(handles[t % R], x[t], 1, tau_x, tau_s[t % R], y[t], stream=cs)
+            thr_us = timed_graph(thr_step, reps=5)
+            tok = s1h = s2h = eh = 0.0
+            for h in handles:
+                a_, b_, c_, d_ = pb.prox_runtime_sparsity(h)
+                tok += a_; s1h += a_ * b_; s2h += a_ * c_; eh += a_ * d_
+            threshold_mode = {"us_per_call": thr_us / T if thr_us else None, "tau_x": tau_x,
+                              "tau_s_mean": float(np.mean(tau_s)), "calibration_tokens": ncal,
+                              "s1_hat": s1h / max(tok, 1), "s2_hat": s2h / max(tok, 1), "e_hat": eh / max(tok, 1),
+                              "target": {"s1": s1_t, "s2": s2_t, "e": E_PCT / 100.0}}
+        except Exception as ex:                        # pragma: no cover
+            sys.stderr.write(f"threshold-mode measurement failed: {ex}\n")
+
         # Proxy-cost ratio alpha (appendix "Empirical Proxy-Cost Ratios"): latency of the integer proxy
         # GEMV over that of the 16-bit GEMV at the same input sparsity, both by the step-wise kernel,
         # every call on another weight replica (cold HBM).
@@ -532,6 +569,7 @@ def run_prox(args):
             "dense_cublas_bf16_us_per_call": dense_us,
             "batch8": batch8,
             "decode_stack": decode_stack,
+            "threshold_mode": threshold_mode,
             "alpha": alpha,
             "clocks": clocks,
         }

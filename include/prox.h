@@ -222,6 +222,11 @@ prox_status_t prox_stage1_mask_threshold(prox_ffn_t* h, const void* x_dev, int B
                                          float* scores_dev_or_null, void* stream);
 prox_status_t prox_stage2_ffn_var(prox_ffn_t* h, const void* x_dev, int B, const int32_t* sel_dev,
                                   const int32_t* count_dev, void* y_dev, void* stream);
+/* prox_ffn_forward_threshold at B = 1 is one launch of the persistent kernel in
+ * its threshold form (no k-th element search); the mask it used can be read with
+ * prox_ffn_last_mask(h, 1, n, ...) where n is the kept-channel count that
+ * prox_runtime_sparsity reports, and is ascending.  Otherwise it is
+ * prox_stage1_mask_threshold followed by prox_stage2_ffn_var. */
 prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x_dev, int B, float tau_x,
                                          float tau_s, void* y_dev, void* stream);
 

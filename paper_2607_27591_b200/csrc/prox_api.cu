@@ -475,7 +475,7 @@ struct FusedPlan {
   size_t smem;
 };
 
-FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
+FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   FusedPlan pl;
   std::memset(&pl, 0, sizeof(pl));
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
@@ -492,6 +492,11 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;      // reduction scratch
   if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
   if ((k2 + G - 1) / G + 2 > kMySelCap) return pl;       // a block's share: definite part + part of the threshold bin
+  if (thresh) {
+    // any number of channels may pass the threshold: a block's share of all of them must fit, the scores
+    // must fit in shared memory (no radix fallback in this form), counts are kept in 16 bits
+    if ((F + G - 1) / G + 2 > kMySelCap || (size_t)F * 4 + 256 > (size_t)pl.big_bytes || F >= 65536) return pl;
+  }
   pl.nstrips = nstrips_for(F, h->bits);
   // row split: fill the grid evenly (items = strips * ksplit run in rounds of G blocks)
   int best = 1;
@@ -512,10 +517,10 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2) {
   return pl;
 }
 
-template <int BITS, int NG, bool NORM>
+template <int BITS, int NG, bool NORM, bool THRESH>
 cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
   static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
-  auto kern = prox_fused_kernel<BITS, NG, NORM>;
+  auto kern = prox_fused_kernel<BITS, NG, NORM, THRESH>;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
@@ -537,7 +542,9 @@ cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStr
 
 template <int BITS, int NG>
 cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
-  return prm.xres ? launch_fused_tn<BITS, NG, true>(pl, prm, st) : launch_fused_tn<BITS, NG, false>(pl, prm, st);
+  if (prm.count_out) return launch_fused_tn<BITS, NG, false, true>(pl, prm, st);      // threshold form
+  return prm.xres ? launch_fused_tn<BITS, NG, true, false>(pl, prm, st)
+                  : launch_fused_tn<BITS, NG, false, false>(pl, prm, st);
 }
 
 // 1/d_model and eps as pairs of floats for the device-side RMSNorm
@@ -551,7 +558,8 @@ RmsConst rms_const(int D, double eps) {
 
 prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int k1, int k2, void* y,
                            int* sel_out, cudaStream_t st, const float* xres = nullptr,
-                           const uint16_t* norm_w = nullptr, double eps = 0.0, float* xres_out = nullptr) {
+                           const uint16_t* norm_w = nullptr, double eps = 0.0, float* xres_out = nullptr,
+                           const float* taus = nullptr) {
   FusedParams prm;
   std::memset(&prm, 0, sizeof(prm));
   prm.P = h->P; prm.S = h->S; prm.wg = h->wg; prm.wu = h->wu; prm.wdt = h->wdt;
@@ -567,6 +575,14 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.big_bytes = pl.big_bytes; prm.nslots = pl.nslots;
   prm.trace = h->trace;
   prm.xres = xres; prm.norm_w = norm_w; prm.rc = rms_const(h->cfg.d_model, eps); prm.xres_out = xres_out;
+  if (taus) {
+    // |x| >= tau_x  <=>  15-bit bf16 magnitude >= ceil(bits(tau_x) / 2^16);  score >= tau_s  <=>  bits >= bits
+    uint32_t bx, bs;
+    std::memcpy(&bx, &taus[0], 4); std::memcpy(&bs, &taus[1], 4);
+    prm.tkey_x = (bx >> 16) + ((bx & 0xffffu) ? 1u : 0u);
+    prm.tkey_s = bs;
+    prm.cnt_x_out = h->cnt_x; prm.count_out = h->cnt_s; prm.counters = h->counters;
+  }
   cudaError_t e;
   {
     LaunchScope ls(h, kKFused, st);
@@ -1012,6 +1028,17 @@ prox_status_t prox_stage2_ffn_var(prox_ffn_t* h, const void* x, int B, const int
 prox_status_t prox_ffn_forward_threshold(prox_ffn_t* h, const void* x, int B, float tau_x, float tau_s,
                                          void* y, void* stream) {
   if (!h) return PROX_ERR_INVALID_ARG;
+  if (B == 1 && h->quantized && x && y && aligned16(x) && aligned16(y) && tau_x >= 0.f && tau_s >= 0.f &&
+      tau_x < INFINITY && tau_s < INFINITY) {
+    // one launch of the persistent kernel in its threshold form
+    const FusedPlan pl = plan_fused(h, h->cfg.d_model, h->cfg.d_ff, true);
+    if (pl.ok) {
+      const float taus[2] = {tau_x, tau_s};
+      h->sel_unordered = 0;
+      return launch_fused(h, pl, x, h->cfg.d_model, h->cfg.d_ff, y, h->sel, static_cast<cudaStream_t>(stream),
+                          nullptr, nullptr, 0.0, nullptr, taus);
+    }
+  }
   prox_status_t s = prox_stage1_mask_threshold(h, x, B, tau_x, tau_s, h->sel, h->cnt_s, nullptr, stream);
   if (s != PROX_OK) return s;
   return prox_stage2_ffn_var(h, x, B, h->sel, h->cnt_s, y, stream);

@@ -62,6 +62,11 @@ struct FusedParams {
   // Layer sub-block form (all NULL / 0 otherwise): the input is bf16(RMSNorm(xres) * norm_w) and the
   // result is xres + y, written as fp32 to xres_out (which may be xres itself).
   const float* xres; const uint16_t* norm_w; float* xres_out; RmsConst rc;
+  // Threshold form (THRESH): keep |x_i| >= tau_x and score_j >= tau_s instead of the k1 / k2 largest.
+  // tkey_x = smallest 15-bit bf16 magnitude that is >= tau_x, tkey_s = bits of tau_s (scores are >= 0, so
+  // their bit patterns order like their values).  Counts go to cnt_x_out / count_out and into counters.
+  unsigned tkey_x, tkey_s;
+  int* cnt_x_out; int* count_out; unsigned long long* counters;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -266,15 +271,17 @@ struct FusedSmem {
 };
 
 // NG = warp groups of the down projection (4: d_model <= 4096, 2: <= 8192, 1: <= 16384)
-// NORM = layer sub-block form (RMSNorm in the prologue, residual add at the end): an instantiation of its
-// own, so that the plain call carries none of its code or registers.
-template <int BITS, int NG, bool NORM = false>
+// NORM = layer sub-block form (RMSNorm in the prologue, residual add at the end); THRESH = threshold
+// form of the two masks (Sec. 4.1 indicators with calibrated thresholds; no k-th element search at all).
+// Instantiations of their own, so that the plain call carries none of their code or registers.
+template <int BITS, int NG, bool NORM = false, bool THRESH = false>
 __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const FusedParams p) {
   constexpr int CH = ProxyFmt<BITS>::CH, NACC = ProxyFmt<BITS>::NACC;
   constexpr int NT = kFusedThreads;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   FusedSmem& sm = *reinterpret_cast<FusedSmem*>(smem_raw);
-  const int D = p.D, F = p.F, k1 = p.k1, k2 = p.k2;
+  const int D = p.D, F = p.F, k2 = p.k2;
+  int k1 = p.k1;                         // THRESH: becomes the number of kept inputs after phase A
   uint16_t* xs = reinterpret_cast<uint16_t*>(smem_raw + ((sizeof(FusedSmem) + 127) & ~size_t(127)));
   uint16_t* idx16 = xs + D;
   float* xf = reinterpret_cast<float*>(idx16 + D);
@@ -357,9 +364,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   // ------------------------------------------------- A: input mask (top-k1 of |x|)
   {
     const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
-    const bool all = k1 >= D;
+    const bool all = THRESH ? (p.tkey_x == 0u) : (k1 >= D);
     unsigned T = 0, quota = 0;
-    if (!all) {
+    if (THRESH) {
+      T = p.tkey_x - 1u;                 // kept: key > T, i.e. |x| >= tau_x; no ties to ration
+    } else if (!all) {
       // level 1: the top 10 of the 15 key bits; level 2: the other 5
 #pragma unroll 1
       for (int i = tid; i < D / 2; i += NT) {
@@ -407,6 +416,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     if (lane == 31) sm.wsum[warp] = inc;
     __syncthreads();
     PROX_TRACE(14);
+    if (THRESH) {
+      k1 = (int)__reduce_add_sync(0xffffffffu, (lane < kFusedWarps) ? (sm.wsum[lane] & 0xffffu) : 0u);
+      if (cta == 0 && tid == 0) {
+        if (p.cnt_x_out) p.cnt_x_out[0] = k1;
+        if (p.counters) { atomicAdd(p.counters, 1ull); atomicAdd(p.counters + 1, (unsigned long long)k1); }
+      }
+    }
     {
       const unsigned ex = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u) + inc - cnt;
       unsigned rg = ex & 0xffffu, re = ex >> 16;
@@ -660,7 +676,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     auto key4_at = [&](int i) -> uint4 {                  // i % 4 == 0
       return in_smem ? lds128(skey_u32 + (uint32_t)i * 4u) : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
     };
-    if (tid < 512) cp_async16(smem_u32(sm.hist) + (uint32_t)tid * 16u, p.ghist + tid * 4);
+    if (!THRESH && tid < 512) cp_async16(smem_u32(sm.hist) + (uint32_t)tid * 16u, p.ghist + tid * 4);
     cp_async_commit();
     if (in_smem) {
 #pragma unroll 1
@@ -671,10 +687,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     cp_async_wait<1>();                                    // the histogram (the keys may still be on their way)
     consumer_sync();
     PROX_TRACE(16);
-    unsigned nd;                                           // channels above bin b1
-    const unsigned b1 = kth_in_block<4, true>(sm.hist, (unsigned)k2, sm.wsum, lane, warp, &nd);
-    const unsigned kk = (unsigned)k2 - nd;                 // members of b1 to keep (>= 1)
-    const unsigned nb1 = sm.hist[b1];
+    unsigned nd = 0;                                       // channels above bin b1 (THRESH: at or above tau_s)
+    unsigned b1 = 0, kk = 0, nb1 = 0;
+    if (!THRESH) {
+      b1 = kth_in_block<4, true>(sm.hist, (unsigned)k2, sm.wsum, lane, warp, &nd);
+      kk = (unsigned)k2 - nd;                              // members of b1 to keep (>= 1)
+      nb1 = sm.hist[b1];
+    }
     uint32_t list_u32 = smem_u32(idx16);                   // 2 * D bytes: room for D / 4 members
     uint32_t list_off = 0;                                 // offset in the big buffer when it has to go there
     bool list_in_big = false;
@@ -693,10 +712,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     consumer_sync();                                       // the keys are there for everyone; wsum is free again
     if (staged) {
       // k2 * G < 2^31 is checked on the host, so the share bounds fit 32 bits
-      const int Rd0 = (int)((nd * (unsigned)cta) / (unsigned)G), Rc0 = (int)((kk * (unsigned)cta) / (unsigned)G);
-      const int ndm = min((int)((nd * (unsigned)(cta + 1)) / (unsigned)G) - Rd0, kMySelCap);
-      const int ncm = min((int)((kk * (unsigned)(cta + 1)) / (unsigned)G) - Rc0, kMySelCap - ndm);
-      const int Rd1 = Rd0 + ndm, Rc1 = Rc0 + ncm;
+      // (THRESH: nd is only known after the counting pass; the bounds are set there)
+      int Rd0 = (int)((nd * (unsigned)cta) / (unsigned)G);
+      const int Rc0 = (int)((kk * (unsigned)cta) / (unsigned)G);
+      int ndm = min((int)((nd * (unsigned)(cta + 1)) / (unsigned)G) - Rd0, kMySelCap);
+      const int ncm = THRESH ? 0 : min((int)((kk * (unsigned)(cta + 1)) / (unsigned)G) - Rc0, kMySelCap - ndm);
+      int Rd1 = Rd0 + ndm;
+      const int Rc1 = Rc0 + ncm;
       n_mine = ndm + ncm;
       // pass 1: a consumer thread owns a run of 4-channel groups and counts its definite
       // channels and its members of b1 (packed in one word); one warp scan, warp totals
@@ -714,9 +736,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         unsigned d4 = 0, c4 = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const unsigned bin = k4[e] >> 20;
-          d4 |= ((bin > b1) ? 1u : 0u) << e;
-          c4 |= ((bin == b1) ? 1u : 0u) << e;
+          if (THRESH) {
+            d4 |= ((k4[e] >= p.tkey_s) ? 1u : 0u) << e;
+          } else {
+            const unsigned bin = k4[e] >> 20;
+            d4 |= ((bin > b1) ? 1u : 0u) << e;
+            c4 |= ((bin == b1) ? 1u : 0u) << e;
+          }
         }
         cnt += (unsigned)__popc(d4) | ((unsigned)__popc(c4) << 16);
         if (masks) {
@@ -726,6 +752,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       }
       const unsigned inc = warp_scan_incl(cnt, lane);
       if (lane == 31) sm.wsum[warp] = inc;
+      if (THRESH) {
+        consumer_sync();                                   // the warps' totals: how many channels are kept
+        nd = __reduce_add_sync(0xffffffffu, (lane < kFusedConsumerWarps) ? (sm.wsum[lane] & 0xffffu) : 0u);
+        Rd0 = (int)((nd * (unsigned)cta) / (unsigned)G);
+        ndm = min((int)((nd * (unsigned)(cta + 1)) / (unsigned)G) - Rd0, kMySelCap);
+        Rd1 = Rd0 + ndm;
+        n_mine = ndm;
+        if (cta == 0 && tid == 0) {
+          if (p.count_out) p.count_out[0] = (int)nd;
+          if (p.counters) atomicAdd(p.counters + 2, (unsigned long long)nd);
+        }
+      }
       if (tid == 0) {
         const uint32_t rb = (uint32_t)D * 2u;
         sm.keys_s0 = (int)(key_off / rb); sm.keys_s1 = (int)((key_off + (uint32_t)F * 4u + rb - 1u) / rb);
@@ -760,7 +798,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             const unsigned k4[4] = {kv.x, kv.y, kv.z, kv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              if ((k4[e] >> 20) > b1) {
+              if (THRESH ? (k4[e] >= p.tkey_s) : ((k4[e] >> 20) > b1)) {
                 if (dpos >= Rd0 && dpos < Rd1) {
                   sm.mysel[dpos - Rd0] = q * 4 + e;
                   if (p.sel_out) p.sel_out[dpos] = q * 4 + e;

@@ -447,6 +447,56 @@ def test_threshold_variant(pb, toy):
     assert torch.allclose(y, y2, rtol=0, atol=1e-5 * float(y.abs().max()))
 
 
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0)])
+def test_threshold_forward_in_one_launch(pb, toy, bits, group):
+    """prox_ffn_forward_threshold at batch 1 is the persistent kernel in its threshold form: masks by
+    |x| >= tau_x and score >= tau_s (Sec. 4.1 indicators), counts vary per token."""
+    wl, p = toy
+    dg, du, _ = p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    launches = 0
+    for t in (0, 3, 11, 20):
+        mags = np.sort(np.abs(p.x[t]))[::-1]
+        for tau_x, frac in ((float(mags[k1 - 1]), 0.3), (0.0, 0.6), (float(mags[5]), 0.05)):
+            idx_t = po.input_threshold(p.x[t], np.float32(tau_x))
+            score_t = po.proxy_scores(p.x[t], idx_t, dg, du)
+            srt = np.sort(score_t)[::-1]
+            kk = max(1, int(frac * p.F))
+            tau_s = float(np.float32((srt[kk - 1] + srt[kk]) / 2))
+            sel_t = po.channel_threshold(score_t, tau_s)
+            y = p.y_empty()
+            pb.prox_runtime_sparsity(p.h, reset=True)
+            l0 = pb.prox_launch_count(p.h)
+            pb.prox_ffn_forward_threshold(p.h, p.t_x[t], 1, tau_x, tau_s, y)
+            launches = pb.prox_launch_count(p.h) - l0
+            torch.cuda.synchronize()
+            tok, s1h, s2h, _ = pb.prox_runtime_sparsity(p.h)
+            n_in, n = int(round((1 - s1h) * p.D)), int(round((1 - s2h) * p.F))
+            assert tok == 1 and n_in == len(idx_t), (n_in, len(idx_t))
+            got = np.empty(0, dtype=np.int64)
+            if n > 0:
+                used = torch.empty(1, n, dtype=torch.int32, device="cuda")
+                pb.prox_ffn_last_mask(p.h, 1, n, used)
+                got = used.cpu().numpy()[0].astype(np.int64)
+                assert np.all(got[1:] > got[:-1])
+            near = np.abs(score_t - tau_s) <= 1e-3 * tau_s
+            assert np.all(near[np.setxor1d(got, sel_t)])
+            y_ref, _ = po.stage2(p.x[t], got, p.wg, p.wu, p.wd)
+            check_y(y.cpu().numpy()[0], y_ref, extra_abs=1e-30)
+    assert launches == 1
+    # nothing passes tau_x: all scores are 0; with tau_s = 0 every channel passes and y is the dense FFN
+    y = p.y_empty()
+    pb.prox_ffn_forward_threshold(p.h, p.t_x[2], 1, 1e30, 0.0, y)
+    torch.cuda.synchronize()
+    y_dense, _ = po.dense_ffn(p.x[2], p.wg, p.wu, p.wd)
+    check_y(y.cpu().numpy()[0], y_dense)
+    # nothing passes tau_s: y = 0
+    pb.prox_ffn_forward_threshold(p.h, p.t_x[2], 1, 0.5, 1e30, y)
+    torch.cuda.synchronize()
+    assert float(y.abs().max()) == 0.0
+    assert pb.prox_last_device_status(p.h) == 0
+
+
 # ------------------------------------------------------------- pack save/load
 # ------------------------------------------------------------ ablation forms
 @pytest.mark.parametrize("B", [1, 3, 8])
