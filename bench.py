@@ -454,6 +454,46 @@ def run_prox(args):
         except Exception as ex:                        # pragma: no cover
             sys.stderr.write(f"threshold-mode measurement failed: {ex}\n")
 
+        # The same 36-layer loop with thresholded masks (per-layer thresholds calibrated on the streams of
+        # the first tokens: tau_x over |FFN input| at level s1, tau_s over the proxy scores at level s2).
+        try:
+            ncal = 8
+            s1_t, s2_t = 1.0 - k1 / D, 1.0 - k2 / F
+            tr = torch.empty(ncal, LAYERS + 1, D, dtype=torch.float32, device=dev)
+            for i in range(ncal):
+                xi = x[i:i + 1].float().contiguous()
+                pb.prox_ffn_stack_forward(stack_handles, nw, 1e-6, xi, 1, k1, k2, tr[i], stream=sp)
+            stream.synchronize()
+            ltx, lts = [], []
+            scl = torch.empty(ncal, F, dtype=torch.float32, device=dev)
+            sel_l = torch.empty(1, F, dtype=torch.int32, device=dev)
+            cnt_l = torch.empty(1, dtype=torch.int32, device=dev)
+            for l in range(LAYERS):
+                xin = tr[:, l, :]
+                xn = (xin * torch.rsqrt((xin * xin).mean(dim=1, keepdim=True) + 1e-6) * nw[l].float()).to(torch.bfloat16)
+                ltx.append(float(torch.quantile(xn.float().abs().flatten(), s1_t)))
+                for i in range(ncal):
+                    pb.prox_stage1_mask_threshold(stack_handles[l], xn[i], 1, ltx[-1], 0.0, sel_l, cnt_l, scl[i], stream=sp)
+                stream.synchronize()
+                lts.append(float(torch.quantile(scl.flatten(), s2_t)))
+            for h in handles:
+                pb.prox_runtime_sparsity(h, reset=True)
+
+            def stack_thr_step():
+                xr.copy_(xr0)
+                pb.prox_ffn_stack_forward_threshold(stack_handles, nw, 1e-6, xr, 1, ltx, lts, None,
+                                                    stream=torch.cuda.current_stream().cuda_stream)
+            st_us = timed_graph(stack_thr_step, reps=10)
+            tok = eh = 0.0
+            for h in handles:
+                a_, b_, c_, d_ = pb.prox_runtime_sparsity(h)
+                tok += a_; eh += a_ * d_
+            decode_stack["threshold_form"] = {"ms_per_token": st_us / 1e3 if st_us else None,
+                                              "us_per_layer": st_us / LAYERS if st_us else None,
+                                              "e_hat": eh / max(tok, 1), "calibration_tokens": ncal}
+        except Exception as ex:                        # pragma: no cover
+            sys.stderr.write(f"threshold decode loop failed: {ex}\n")
+
         # Proxy-cost ratio alpha (appendix "Empirical Proxy-Cost Ratios"): latency of the integer proxy
         # GEMV over that of the 16-bit GEMV at the same input sparsity, both by the step-wise kernel,
         # every call on another weight replica (cold HBM).

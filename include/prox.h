@@ -269,6 +269,17 @@ prox_status_t prox_ffn_stack_forward(prox_ffn_t* const* layers, int n_layers, co
                                      double eps, float* x_res_dev, int B, int k1, int k2,
                                      float* trace_dev_or_null, void* stream);
 
+/* The same two calls with the threshold form of the masks (|x_i| >= tau_x,
+ * score_j >= tau_s; per-layer thresholds in host arrays of n_layers floats for
+ * the stack).  At B = 1 a layer is one launch; kept counts go to the handle's
+ * counters (prox_runtime_sparsity). */
+prox_status_t prox_ffn_block_forward_threshold(prox_ffn_t* h, const float* x_res_dev, const void* norm_w_dev,
+                                               double eps, int B, float tau_x, float tau_s,
+                                               float* x_res_out_dev, void* stream);
+prox_status_t prox_ffn_stack_forward_threshold(prox_ffn_t* const* layers, int n_layers, const void* norm_w_dev,
+                                               double eps, float* x_res_dev, int B, const float* tau_x_host,
+                                               const float* tau_s_host, float* trace_dev_or_null, void* stream);
+
 /* Runtime mask counts accumulated by the threshold entry points since the last
  * reset (appendix "Threshold Calibration and Runtime Sparsity":
  * e^ = s2^ - 2 alpha (1 - s1^) / 3).  Host-synchronous.  Any pointer may be NULL. */

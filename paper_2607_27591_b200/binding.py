@@ -55,6 +55,8 @@ _SIGS = {
     "prox_ffn_forward_proxy_values": [_vp, _vp, _i, _i, _i, _vp, _vp],
     "prox_ffn_block_forward": [_vp, _vp, _vp, _d, _i, _i, _i, _vp, _vp],
     "prox_ffn_stack_forward": [C.POINTER(_vp), _i, _vp, _d, _vp, _i, _i, _i, _vp, _vp],
+    "prox_ffn_block_forward_threshold": [_vp, _vp, _vp, _d, _i, _f, _f, _vp, _vp],
+    "prox_ffn_stack_forward_threshold": [C.POINTER(_vp), _i, _vp, _d, _vp, _i, C.POINTER(_f), C.POINTER(_f), _vp, _vp],
     "prox_runtime_sparsity": [_vp, _d, C.POINTER(C.c_int64), C.POINTER(_d), C.POINTER(_d), C.POINTER(_d), _i],
     "prox_allocate_budget": [_d, _d, _d, _d, _d, C.POINTER(_d), C.POINTER(_d)],
     "prox_sparsity_to_k": [_d, _i, C.POINTER(_i)],
@@ -216,6 +218,22 @@ def prox_ffn_stack_forward(handles, norm_w, eps: float, x_res, B: int, k1: int, 
     arr = (_vp * len(handles))(*handles)
     _check(_lib.prox_ffn_stack_forward(arr, len(handles), _ptr(norm_w), eps, _ptr(x_res), B, k1, k2,
                                        _ptr(trace), _ptr(stream)), "prox_ffn_stack_forward")
+
+
+def prox_ffn_block_forward_threshold(handle: int, x_res, norm_w, eps: float, B: int, tau_x: float, tau_s: float,
+                                     x_res_out, stream=None) -> None:
+    _check(_lib.prox_ffn_block_forward_threshold(handle, _ptr(x_res), _ptr(norm_w), eps, B, tau_x, tau_s,
+                                                 _ptr(x_res_out), _ptr(stream)), "prox_ffn_block_forward_threshold")
+
+
+def prox_ffn_stack_forward_threshold(handles, norm_w, eps: float, x_res, B: int, tau_x, tau_s, trace=None,
+                                     stream=None) -> None:
+    n = len(handles)
+    arr = (_vp * n)(*handles)
+    tx = (_f * n)(*[float(v) for v in tau_x])
+    ts = (_f * n)(*[float(v) for v in tau_s])
+    _check(_lib.prox_ffn_stack_forward_threshold(arr, n, _ptr(norm_w), eps, _ptr(x_res), B, tx, ts, _ptr(trace),
+                                                 _ptr(stream)), "prox_ffn_stack_forward_threshold")
 
 
 def prox_runtime_sparsity(handle: int, alpha: float = 1.0 / 3.0, reset: bool = False):

@@ -41,8 +41,8 @@ struct prox_ffn {
   size_t part_floats;
   unsigned* ticket;         // [maxB][nstrips_max]
   float* scores;            // [maxB][F]
-  float* svals;             // [maxB][F] signed proxy values (proxy-values-into-down variant), on first use
-  uint16_t* xn;             // [maxB][D] bf16 FFN input of the layer sub-block form (step-wise path), on first use
+  float* svals;             // [maxB][F] signed proxy values (proxy-values-into-down variant)
+  uint16_t* xn;             // [maxB][D] bf16 FFN input of the layer sub-block form (step-wise path)
   const float* fin_resid;   // while a layer sub-block call is enqueued: the residual stream to add ...
   float* fin_out;           // ... and where the sum goes
   int* sel;                 // [maxB][F]
@@ -542,7 +542,9 @@ cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStr
 
 template <int BITS, int NG>
 cudaError_t launch_fused_t(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
-  if (prm.count_out) return launch_fused_tn<BITS, NG, false, true>(pl, prm, st);      // threshold form
+  if (prm.count_out)                                                                   // threshold form
+    return prm.xres ? launch_fused_tn<BITS, NG, true, true>(pl, prm, st)
+                    : launch_fused_tn<BITS, NG, false, true>(pl, prm, st);
   return prm.xres ? launch_fused_tn<BITS, NG, true, false>(pl, prm, st)
                   : launch_fused_tn<BITS, NG, false, false>(pl, prm, st);
 }
@@ -659,6 +661,8 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   A(dev_alloc(&h->part, h->part_floats));
   A(dev_alloc(&h->ticket, (size_t)MB * ns_max));
   A(dev_alloc(&h->scores, (size_t)MB * F));
+  A(dev_alloc(&h->svals, (size_t)MB * F));      // (allocated here, not on first use: a first use may be under graph capture)
+  A(dev_alloc(&h->xn, (size_t)MB * D));
   A(dev_alloc(&h->sel, (size_t)MB * F));
   A(dev_alloc(&h->cnt_s, (size_t)MB));
   A(dev_alloc(&h->hbuf, (size_t)MB * F));
@@ -835,9 +839,6 @@ prox_status_t prox_ffn_block_forward(prox_ffn_t* h, const float* x_res, const vo
                           static_cast<const uint16_t*>(norm_w), eps, x_res_out);
     }
   }
-  if (!h->xn) {
-    if (dev_alloc(&h->xn, (size_t)h->cfg.max_batch * D) != cudaSuccess) return PROX_ERR_OOM;
-  }
   rmsnorm_kernel<<<B, 256, 0, st>>>(x_res, static_cast<const uint16_t*>(norm_w), rms_const(D, eps), D, h->xn);
   h->launches++;
   CK(cudaGetLastError());
@@ -847,25 +848,72 @@ prox_status_t prox_ffn_block_forward(prox_ffn_t* h, const float* x_res, const vo
   return s;
 }
 
-/* The FFN sub-blocks of consecutive layers applied to one residual stream. */
-prox_status_t prox_ffn_stack_forward(prox_ffn_t* const* layers, int n_layers, const void* norm_w, double eps,
-                                     float* x_res, int B, int k1, int k2, float* trace, void* stream) {
+/* The layer sub-block with the threshold form of the masks. */
+prox_status_t prox_ffn_block_forward_threshold(prox_ffn_t* h, const float* x_res, const void* norm_w, double eps,
+                                               int B, float tau_x, float tau_s, float* x_res_out, void* stream) {
+  prox_status_t s = check_common(h, x_res, B);
+  if (s != PROX_OK) return s;
+  if (!norm_w || !x_res_out || !aligned16(x_res_out) || !aligned16(norm_w)) return PROX_ERR_INVALID_ARG;
+  if (!(eps >= 0.0) || !(tau_x >= 0.f) || !(tau_s >= 0.f) || !(tau_x < INFINITY) || !(tau_s < INFINITY))
+    return PROX_ERR_INVALID_ARG;
+  if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int D = h->cfg.d_model, F = h->cfg.d_ff;
+  if (B == 1) {
+    const FusedPlan pl = plan_fused(h, D, F, true);
+    if (pl.ok) {
+      const float taus[2] = {tau_x, tau_s};
+      h->sel_unordered = 0;
+      return launch_fused(h, pl, nullptr, D, F, nullptr, h->sel, st, x_res, static_cast<const uint16_t*>(norm_w),
+                          eps, x_res_out, taus);
+    }
+  }
+  rmsnorm_kernel<<<B, 256, 0, st>>>(x_res, static_cast<const uint16_t*>(norm_w), rms_const(D, eps), D, h->xn);
+  h->launches++;
+  CK(cudaGetLastError());
+  if ((s = prox_stage1_mask_threshold(h, h->xn, B, tau_x, tau_s, h->sel, h->cnt_s, nullptr, stream)) != PROX_OK) return s;
+  h->fin_resid = x_res; h->fin_out = x_res_out;          // the last kernel adds the residual stream
+  s = launch_stage2(h, h->xn, B, h->sel, F, h->cnt_s, F, nullptr, st);
+  h->fin_resid = nullptr; h->fin_out = nullptr;
+  return s;
+}
+
+/* Stacks of layers: top-k form (tau arrays NULL) or threshold form (one pair of thresholds per layer). */
+static prox_status_t stack_forward(prox_ffn_t* const* layers, int n_layers, const void* norm_w, double eps,
+                                   float* x_res, int B, int k1, int k2, const float* tau_x, const float* tau_s,
+                                   float* trace, void* stream) {
   if (!layers || n_layers < 1 || !norm_w || !x_res) return PROX_ERR_INVALID_ARG;
   for (int l = 0; l < n_layers; ++l) {
     if (!layers[l]) return PROX_ERR_INVALID_ARG;
     if (layers[l]->cfg.d_model != layers[0]->cfg.d_model) return PROX_ERR_INVALID_ARG;
   }
+  if (B < 1 || B > layers[0]->cfg.max_batch) return PROX_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t D = (size_t)layers[0]->cfg.d_model;
   const size_t bytes = (size_t)B * D * sizeof(float);
   if (trace) CK(cudaMemcpyAsync(trace, x_res, bytes, cudaMemcpyDeviceToDevice, st));
   for (int l = 0; l < n_layers; ++l) {
-    const prox_status_t s = prox_ffn_block_forward(layers[l], x_res, static_cast<const uint16_t*>(norm_w) + (size_t)l * D,
-                                                   eps, B, k1, k2, x_res, stream);
+    const uint16_t* nw = static_cast<const uint16_t*>(norm_w) + (size_t)l * D;
+    const prox_status_t s = tau_x
+        ? prox_ffn_block_forward_threshold(layers[l], x_res, nw, eps, B, tau_x[l], tau_s[l], x_res, stream)
+        : prox_ffn_block_forward(layers[l], x_res, nw, eps, B, k1, k2, x_res, stream);
     if (s != PROX_OK) return s;
     if (trace) CK(cudaMemcpyAsync(trace + (size_t)(l + 1) * B * D, x_res, bytes, cudaMemcpyDeviceToDevice, st));
   }
   return PROX_OK;
+}
+
+prox_status_t prox_ffn_stack_forward_threshold(prox_ffn_t* const* layers, int n_layers, const void* norm_w,
+                                               double eps, float* x_res, int B, const float* tau_x_host,
+                                               const float* tau_s_host, float* trace, void* stream) {
+  if (!tau_x_host || !tau_s_host) return PROX_ERR_INVALID_ARG;
+  return stack_forward(layers, n_layers, norm_w, eps, x_res, B, 0, 0, tau_x_host, tau_s_host, trace, stream);
+}
+
+/* The FFN sub-blocks of consecutive layers applied to one residual stream. */
+prox_status_t prox_ffn_stack_forward(prox_ffn_t* const* layers, int n_layers, const void* norm_w, double eps,
+                                     float* x_res, int B, int k1, int k2, float* trace, void* stream) {
+  return stack_forward(layers, n_layers, norm_w, eps, x_res, B, k1, k2, nullptr, nullptr, trace, stream);
 }
 
 // Ablation A3 of Sec. "Ablation Studies": Stage 1 as always, then the selected proxy values themselves
@@ -880,9 +928,6 @@ prox_status_t prox_ffn_forward_proxy_values(prox_ffn_t* h, const void* x, int B,
   if (!h->quantized) return PROX_ERR_NOT_QUANTIZED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
-  if (!h->svals) {
-    if (dev_alloc(&h->svals, (size_t)h->cfg.max_batch * F) != cudaSuccess) return PROX_ERR_OOM;
-  }
   h->sel_unordered = 0;
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, h->scores, st, h->svals)) != PROX_OK) return s;

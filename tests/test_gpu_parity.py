@@ -635,6 +635,67 @@ def test_ffn_stack_forward_layer_by_layer(pb, B):
             q.close()
 
 
+@pytest.mark.parametrize("B", [1, 2])
+def test_ffn_stack_forward_threshold_layer_by_layer(pb, B):
+    """The layer sub-block with thresholded masks (at B = 1 one launch per layer), three layers in place."""
+    from tests.gpu_common import dev_bf16
+    L, D, F = 3, 512, 1536
+    probs = []
+    try:
+        for l in range(L):
+            wg, wu, wd, x = inputs.make_small(D, F, 4, seed=60 + l)
+            probs.append(Problem(pb, wg, wu, wd, x, max_batch=2))
+        deqs = [q.quantize(4, 128) for q in probs]
+        nw_bits = np.stack([_norm_weight(D, 70 + l) for l in range(L)])
+        nw64 = [po.bf16_to_f64(nw_bits[l]) for l in range(L)]
+        t_nw = dev_bf16(nw_bits)
+        eps = 1e-6
+        x0 = (probs[0].x[:B] * 2.0).astype(np.float32)
+        # thresholds from the oracle's own top-k stack of token 0: between the k-th and the next value
+        k1, k2 = 154, 358
+        layers = [(nw64[l], deqs[l][0], deqs[l][1], probs[l].wg, probs[l].wu, probs[l].wd) for l in range(L)]
+        xs = po.ffn_stack(x0[0].astype(np.float64), layers, eps, k1, k2)
+        tau_x, tau_s = [], []
+        for l in range(L):
+            xn = po.bf16_to_f64(po.f64_to_bf16_bits(po.rmsnorm(xs[l], nw64[l], eps)))
+            mags = np.sort(np.abs(xn))[::-1]
+            tau_x.append(float(np.float32(mags[k1 - 1])))
+            sc = np.sort(po.proxy_scores(xn, po.input_threshold(xn, np.float32(tau_x[-1])), deqs[l][0], deqs[l][1]))[::-1]
+            tau_s.append(float(np.float32((sc[k2 - 1] + sc[k2]) / 2)))
+        t_x = torch.from_numpy(x0).cuda()
+        trace = torch.zeros(L + 1, B, D, dtype=torch.float32, device="cuda")
+        l0 = sum(pb.prox_launch_count(q.h) for q in probs)
+        pb.prox_ffn_stack_forward_threshold([q.h for q in probs], t_nw, eps, t_x, B, tau_x, tau_s, trace)
+        torch.cuda.synchronize()
+        if B == 1:
+            assert sum(pb.prox_launch_count(q.h) for q in probs) - l0 == L      # one launch per layer
+        tr = trace.cpu().numpy()
+        assert np.array_equal(tr[0], x0) and np.array_equal(tr[L], t_x.cpu().numpy())
+        for l in range(L):
+            dg, du, _ = deqs[l]
+            for b in range(B):
+                x_in = tr[l, b].astype(np.float64)
+                xn = po.bf16_to_f64(po.f64_to_bf16_bits(po.rmsnorm(x_in, nw64[l], eps)))
+                idx = po.input_threshold(xn, np.float32(tau_x[l]))
+                score = po.proxy_scores(xn, idx, dg, du)
+                sel_t = po.channel_threshold(score, tau_s[l])
+                # y of this layer from the oracle on its own mask; a channel inside the band may differ:
+                # bound the difference by the contribution of the band channels
+                y_ref, s_sp = po.stage2(xn, sel_t, probs[l].wg, probs[l].wu, probs[l].wd)
+                near = np.nonzero(np.abs(score - tau_s[l]) <= 1e-3 * tau_s[l])[0]
+                slack = 0.0
+                if len(near):
+                    _, s_near = po.stage2(xn, near, probs[l].wg, probs[l].wu, probs[l].wd)
+                    slack = float(np.sum(np.abs(s_near)) * np.max(np.abs(probs[l].wd)))
+                check_y(tr[l + 1, b].astype(np.float64) - x_in, y_ref,
+                        extra_abs=slack + float(np.max(np.abs(tr[l + 1, b]))) * 2.0 ** -23)
+        for q in probs:
+            assert pb.prox_last_device_status(q.h) == 0
+    finally:
+        for q in probs:
+            q.close()
+
+
 def test_pack_save_load_roundtrip(pb, toy, tmp_path):
     wl, p = toy
     p.quantize(4, 128)
