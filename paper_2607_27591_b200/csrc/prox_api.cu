@@ -473,6 +473,7 @@ struct FusedPlan {
   bool ok;
   int grid, ksplit, nstrips, big_bytes, nslots, xch;
   size_t smem;
+  int optin;            // the device's opt-in limit: what the kernels' dynamic shared memory attribute is set to
 };
 
 FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
@@ -513,6 +514,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   pl.grid = G;
   pl.xch = D <= 4096 ? 4 : (D <= 8192 ? 2 : 1);          // warp groups of the down projection
   pl.smem = fixed + (size_t)pl.big_bytes;
+  pl.optin = h->smem_optin;
   pl.ok = true;
   return pl;
 }
@@ -522,7 +524,8 @@ cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStr
   static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
   auto kern = prox_fused_kernel<BITS, NG, NORM, THRESH>;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    // the limit, not this plan's size: another handle's shape may need a few bytes more
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.optin);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -953,7 +956,7 @@ prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* inf
       : (pl.xch == 1 ? (const void*)prox_fused_kernel<8, 1> : pl.xch == 2 ? (const void*)prox_fused_kernel<8, 2> : (const void*)prox_fused_kernel<8, 4>);
   cudaFuncAttributes fa;
   CK(cudaFuncGetAttributes(&fa, fn));
-  CK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+  CK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.optin));
   int nb = 0;
   CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kFusedThreads, pl.smem));
   info[1] = pl.grid; info[2] = pl.ksplit; info[3] = (int)pl.smem; info[4] = pl.nslots;
