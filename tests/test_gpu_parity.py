@@ -696,6 +696,63 @@ def test_ffn_stack_forward_threshold_layer_by_layer(pb, B):
             q.close()
 
 
+@pytest.mark.parametrize("D,F,bits,group", [(128, 64, 4, 0), (256, 320, 4, 128), (384, 1984, 8, 0), (1024, 4096, 4, 128),
+                                            (640, 2112, 8, 128)])
+def test_forms_on_odd_shapes(pb, D, F, bits, group):
+    """Threshold form, layer sub-block form and both together on shapes with ragged strips and few channels
+    per block, seeded random budgets."""
+    from tests.gpu_common import dev_bf16
+    wg, wu, wd, x = inputs.make_small(D, F, 4, seed=D + F)
+    p = Problem(pb, wg, wu, wd, x, max_batch=2)
+    try:
+        dg, du, _ = p.quantize(bits, group)
+        rng = np.random.default_rng(D * 7 + F)
+        nw_bits = _norm_weight(D, 3)
+        nw64 = po.bf16_to_f64(nw_bits)
+        t_nw = dev_bf16(nw_bits)
+        for trial in range(4):
+            k1 = int(rng.integers(1, D + 1))
+            k2 = int(rng.integers(1, F + 1))
+            t = trial % 4
+            # layer sub-block, top-k
+            x_res = (p.x[t] * 1.3).astype(np.float32)[None, :]
+            t_x = torch.from_numpy(x_res).cuda()
+            out = torch.empty_like(t_x)
+            used = torch.empty(1, k2, dtype=torch.int32, device="cuda")
+            pb.prox_ffn_block_forward(p.h, t_x, t_nw, 1e-5, 1, k1, k2, out)
+            pb.prox_ffn_last_mask(p.h, 1, k2, used)
+            torch.cuda.synchronize()
+            _check_block(p, dg, du, x_res[0].astype(np.float64), nw64, 1e-5, k1, k2, out.cpu().numpy()[0],
+                         used.cpu().numpy()[0].astype(np.int64))
+            # threshold form on the plain input and on the layer sub-block
+            mags = np.sort(np.abs(p.x[t]))[::-1]
+            tau_x = float(mags[k1 - 1])
+            idx_t = po.input_threshold(p.x[t], np.float32(tau_x))
+            score_t = po.proxy_scores(p.x[t], idx_t, dg, du)
+            srt = np.sort(score_t)[::-1]
+            tau_s = float(np.float32(srt[k2 - 1] if k2 == F else (srt[k2 - 1] + srt[k2]) / 2))
+            sel_t = po.channel_threshold(score_t, tau_s)
+            y = p.y_empty()
+            pb.prox_runtime_sparsity(p.h, reset=True)
+            pb.prox_ffn_forward_threshold(p.h, p.t_x[t], 1, tau_x, tau_s, y)
+            torch.cuda.synchronize()
+            tok, s1h, s2h, _ = pb.prox_runtime_sparsity(p.h)
+            n_in, n = int(round((1 - s1h) * D)), int(round((1 - s2h) * F))
+            assert n_in == len(idx_t)
+            got = np.empty(0, dtype=np.int64)
+            if n > 0:
+                u2 = torch.empty(1, n, dtype=torch.int32, device="cuda")
+                pb.prox_ffn_last_mask(p.h, 1, n, u2)
+                got = u2.cpu().numpy()[0].astype(np.int64)
+            near = np.abs(score_t - tau_s) <= 1e-3 * tau_s
+            assert np.all(near[np.setxor1d(got, sel_t)])
+            y_ref, _ = po.stage2(p.x[t], got, p.wg, p.wu, p.wd)
+            check_y(y.cpu().numpy()[0], y_ref, extra_abs=1e-30)
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
+
+
 def test_pack_save_load_roundtrip(pb, toy, tmp_path):
     wl, p = toy
     p.quantize(4, 128)
