@@ -141,6 +141,7 @@ __device__ __forceinline__ void consumer_sync() {     // the 512 consumer thread
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   if (*abort_flag) return false;
+#pragma unroll 1
   for (unsigned it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 256) __nanosleep(64);
@@ -158,6 +159,7 @@ __device__ __forceinline__ bool slot_wait(uint32_t bar, volatile unsigned* seen,
                                           volatile int* abort_flag) {
   if (use > 0 && *seen < use) {
     bool ok = false;
+#pragma unroll 1
     for (unsigned it = 0; it < kSpinLimit; ++it) {
       if (*seen >= use) { ok = true; break; }
       if (it > 256) __nanosleep(32);
@@ -637,6 +639,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     // the count is reset by the host long before 2^32 calls; the low word is enough for the division
     const unsigned long long target = old - (unsigned long long)((unsigned)old % (unsigned)G) + (unsigned long long)G;
     bool ok = (old + 1ull == target);
+#pragma unroll 1
     for (unsigned it = 0; !ok && it < kSpinLimit; ++it) {
       unsigned long long cur;
       asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(cur) : "l"(p.bar_count) : "memory");
@@ -1045,6 +1048,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     if (lane == 0 && alive) {
       // wait (bounded) until the consumer warps have listed the block's definite share
       bool go = false;
+#pragma unroll 1
       for (unsigned it = 0; it < kSpinLimit; ++it) {
         if (*reinterpret_cast<volatile int*>(&sm.go)) { go = true; break; }
         if (*abortp) break;
@@ -1076,6 +1080,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
               return mi >= ready || (!kdone && slot >= ks0 && slot < ks1) || (!cdone && slot >= ls0 && slot < ls1);
             };
             if (blocked()) {
+#pragma unroll 1
               for (unsigned it = 0; it < kSpinLimit; ++it) {
                 ready = *reinterpret_cast<volatile int*>(&sm.nready);
                 kdone = *reinterpret_cast<volatile int*>(&sm.keys_done) != 0;
@@ -1221,6 +1226,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       const unsigned first = issued > (unsigned)NS ? issued - (unsigned)NS : 0u;
       for (unsigned q = first; q < issued; ++q) {        // the latest use of every slot
         const uint32_t bar = smem_u32(&sm.mbar_full[q % (unsigned)NS]);
+#pragma unroll 1
         for (unsigned it = 0; it < 8192u; ++it) {
           if (mbar_try_wait(bar, (q / (unsigned)NS) & 1u)) break;
           __nanosleep(256);
