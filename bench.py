@@ -584,6 +584,13 @@ def run_prox(args):
         us, n = time_oracle(po, ks, mats, xs, args.cpu_seconds, 256)
         cpu = {"value": us, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": f"{n} tokens of the same workload (oracle forward per token, proxies pre-quantized)"}
+        try:                                           # the same on one core (a third of the time budget)
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                us1, n1 = time_oracle(po, ks, mats, xs, args.cpu_seconds / 3.0, 64)
+            cpu["one_core"] = {"value": us1, "unit": UNIT, "cores": 1, "sample": f"{n1} tokens"}
+        except Exception as ex:                        # pragma: no cover
+            sys.stderr.write(f"one-core oracle timing skipped: {ex}\n")
 
     if rank == 0:
         out = {
