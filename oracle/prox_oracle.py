@@ -38,7 +38,7 @@ __all__ = [
     "dequantize", "input_topk", "input_threshold", "input_sparse_projection", "proxy_scores", "channel_topk",
     "channel_threshold", "stage2", "forward", "forward_batch", "allocate_budget",
     "sparsity_to_k", "effective_sparsity", "proxy_values", "forward_proxy_values",
-    "rmsnorm", "ffn_block", "ffn_stack",
+    "rmsnorm", "ffn_block", "ffn_stack", "forward_batch_shared",
 ]
 
 
@@ -277,6 +277,26 @@ def ffn_stack(x_res, layers, eps: float, k1: int, k2: int):
     for (nw, dg, du, wg, wu, wd) in layers:
         xs.append(ffn_block(xs[-1], nw, eps, k1, k2, dg, du, wg, wu, wd)[0])
     return xs
+
+
+# ------------------------------------------------- a batch with one shared mask
+def forward_batch_shared(xs, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down):
+    """A batch policy beyond the paper (it treats single-batch decoding only and
+    names batching as future work): every token keeps its own input mask and
+    its own proxy scores, the batch keeps ONE channel mask, the k2 channels of
+    largest summed score  sum_b |s~_{b,j}|  (ties to the lower channel), and
+    Stage 2 of every token runs on that mask.  With one token this is `forward`.
+    Returns (sel, threshold, shared score, list of y per token)."""
+    scores = []
+    for x in xs:
+        idx_x = input_topk(x, k1)
+        scores.append(proxy_scores(x, idx_x, deq_gate, deq_up))
+    shared = np.zeros_like(scores[0])
+    for sc in scores:                 # token after token
+        shared = shared + sc
+    sel, thr = channel_topk(shared, k2)
+    ys = [stage2(x, sel, w_gate, w_up, w_down)[0] for x in xs]
+    return sel, thr, shared, ys
 
 
 # ---------------------------------------------------------- budget helper

@@ -546,3 +546,32 @@ def test_ffn_stack_chains_blocks():
     a, _, _ = po.ffn_block(x[1], nw, 1e-6, 50, 70, wg, wu, wg, wu, wd)
     b, _, _ = po.ffn_block(a, nw, 1e-6, 50, 70, wu, wg, wu, wg, wd)
     assert np.array_equal(xs[1], a) and np.array_equal(xs[2], b)
+
+
+# ----------------------------------------------------- shared batch mask pins
+def test_shared_mask_batch_reduces_to_single_token_and_ignores_token_order():
+    wg, wu, wd, x = _problem(seed=31, n_tok=3)
+    dg = po.dequantize(*po.quantize_proxy(wg, 4, 0), 0)
+    du = po.dequantize(*po.quantize_proxy(wu, 4, 0), 0)
+    k1, k2 = 70, 90
+    one = po.forward(x[0], k1, k2, dg, du, wg, wu, wd)
+    sel, thr, shared, ys = po.forward_batch_shared(x[:1], k1, k2, dg, du, wg, wu, wd)
+    assert np.array_equal(sel, one["sel"]) and np.array_equal(ys[0], one["y"]) and thr == one["threshold"]
+    # the same token twice: the sums double, the mask stays
+    sel2, _, shared2, ys2 = po.forward_batch_shared(np.stack([x[0], x[0]]), k1, k2, dg, du, wg, wu, wd)
+    assert np.array_equal(sel2, one["sel"]) and np.array_equal(shared2, 2 * one["score"])
+    # three tokens: mask = full sort of the summed scores, unchanged by the order of the tokens,
+    # and every token's y is Stage 2 on that mask (dense with the other channels zeroed)
+    sel3, thr3, shared3, ys3 = po.forward_batch_shared(x, k1, k2, dg, du, wg, wu, wd)
+    ref = sum(po.proxy_scores(x[b], po.input_topk(x[b], k1), dg, du) for b in (2, 0, 1))
+    np.testing.assert_allclose(shared3, ref, rtol=1e-14)
+    assert np.array_equal(sel3, np.sort(np.argsort(-shared3, kind="stable")[:k2]))
+    selp, _, _, ysp = po.forward_batch_shared(x[::-1], k1, k2, dg, du, wg, wu, wd)
+    assert np.array_equal(selp, sel3)
+    for b in range(3):
+        xt = torch.from_numpy(x[b])
+        s_full = (torch.from_numpy(wu) @ xt) * torch.nn.functional.silu(torch.from_numpy(wg) @ xt)
+        m = torch.zeros(wg.shape[0], dtype=torch.float64)
+        m[torch.from_numpy(sel3)] = 1.0
+        np.testing.assert_allclose(ys3[b], (torch.from_numpy(wd) @ (s_full * m)).numpy(), rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(ysp[2 - b], ys3[b], rtol=0, atol=0)
