@@ -396,9 +396,15 @@ def run_prox(args):
                 torch.matmul(torch.nn.functional.silu(xb @ wg.t()) * (xb @ wu.t()), wd.t(), out=y8[c % 8])
         b8_us = timed_graph(prox8_step)
         d8_us = timed_graph(dense8_step)
+        for h in handles:
+            pb.prox_ffn_set_mask_policy(h, 1)          # one channel mask for the batch (summed scores)
+        s8_us = timed_graph(prox8_step)
+        for h in handles:
+            pb.prox_ffn_set_mask_policy(h, 0)
         batch8 = {"batch": B8, "prox_us_per_call": b8_us / calls8 if b8_us else None,
                   "dense_cublas_bf16_us_per_call": d8_us / calls8 if d8_us else None,
-                  "masks": "per token; weights read once for the union"}
+                  "masks": "per token; weights read once for the union",
+                  "shared_mask_us_per_call": s8_us / calls8 if s8_us else None}
 
         # The FFN sub-blocks of a 36-layer decoder applied to one residual stream, one graph per token
         # (RMSNorm + Prox FFN + residual add per layer in one launch each; layer l reads replica l mod R).

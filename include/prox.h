@@ -132,6 +132,15 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x_dev, int B, int k1, 
  * prox_last_device_status reports bit 4. */
 prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
 
+/* Mask policy of calls with B > 1 (the paper treats batch 1 only and names batching as future work):
+ *   0  every token its own channel mask (default; a token's result is the one it would get alone)
+ *   1  one channel mask for the batch: the k2 channels of largest summed proxy score
+ *      sum_b |s~_{b,j}| (ties: lower channel); input masks and proxy scores stay per token, and
+ *      Stage 2 reads k2 rows instead of the union of B masks.  Built by the tensor-core batch
+ *      path (4-bit proxies); other configurations return UNSUPPORTED from the forward calls.
+ * B = 1 is not affected.  Errors: INVALID_ARG. */
+prox_status_t prox_ffn_set_mask_policy(prox_ffn_t* h, int policy);
+
 /* For B > 1 every token keeps its own masks (the paper covers B = 1 only), and the
  * weights are read once per call for the UNION of the tokens' kept inputs and of
  * their kept channels; a token contributes zero outside its own masks, so its

@@ -70,6 +70,7 @@ _SIGS = {
     "prox_launch_count": [_vp, C.POINTER(C.c_int64)],
     "prox_ffn_set_fused": [_vp, _i],
     "prox_ffn_set_union": [_vp, _i],
+    "prox_ffn_set_mask_policy": [_vp, _i],
     "prox_fused_trace": [_vp, _i, _vp, _i],
     "prox_fused_kernel_info": [_vp, _i, _i, C.POINTER(C.c_int32)],
     "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
@@ -160,6 +161,10 @@ def prox_stage2_ffn_noalloc(x, w_gate, w_up, w_down_t, d_model: int, d_ff: int, 
 
 def prox_ffn_set_fused(handle: int, on: int) -> None:
     _check(_lib.prox_ffn_set_fused(handle, int(on)), "prox_ffn_set_fused")
+
+
+def prox_ffn_set_mask_policy(handle: int, policy: int) -> None:
+    _check(_lib.prox_ffn_set_mask_policy(handle, int(policy)), "prox_ffn_set_mask_policy")
 
 
 def prox_ffn_set_union(handle: int, on: int) -> None:

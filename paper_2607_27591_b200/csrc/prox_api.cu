@@ -68,6 +68,7 @@ struct prox_ffn {
   float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
   int use_mma;              // batch > 1: Stage 2 and the 4-bit proxy GEMM run on the tensor cores
   float* pacc;              // [F / 64][128 code columns][8] proxy sums of the tensor-core batch path, kept at zero
+  int mask_policy;          // batch > 1: 0 = every token its own channel mask, 1 = one mask from the summed scores
   int cmask_marked;         // Stage 1 of the running forward call has set the tokens' bits in cmask already
   unsigned* cmask;          // [F / 4] one byte per channel: which tokens kept it (kept at zero between calls)
   uint8_t* umask;           // [F] that byte for every union row
@@ -342,16 +343,28 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
       proxy_mma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
     }
     CK(cudaGetLastError());
+    if (h->mask_policy == 1) {
+      if (!fast_masks) return PROX_ERR_UNSUPPORTED;
+      LaunchScope ls(h, kKChannel, st);
+      shared_score_kernel<<<(F + 255) / 256, 256, 0, st>>>(scores, B, F, h->svals);
+      batch_channel_mask_kernel<<<1, kFusedThreads, (size_t)F * 4, st>>>(h->svals, F, k2, sel, sel_stride,
+                                                                        mark_mask ? h->cmask : nullptr, (1u << B) - 1u);
+      replicate_mask_kernel<<<(k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B);
+      CK(cudaGetLastError());
+      if (mark_mask) h->cmask_marked = 1;
+      return PROX_OK;
+    }
     if (!fast_masks) return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
     {
       LaunchScope ls(h, kKChannel, st);
       batch_channel_mask_kernel<<<B, kFusedThreads, (size_t)F * 4, st>>>(scores, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr);
+                                                                        mark_mask ? h->cmask : nullptr, 0u);
     }
     CK(cudaGetLastError());
     if (mark_mask) h->cmask_marked = 1;
     return PROX_OK;
   }
+  if (h->mask_policy == 1) return PROX_ERR_UNSUPPORTED;      // the shared mask is built by the tensor-core path only
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_union(h, h->idx_x, D, nullptr, k1, B, D, x, h->u_in, h->u_cnt, h->xu, st)) != PROX_OK) return s;
   const int ns = nstrips_for(F, h->bits);
@@ -608,6 +621,7 @@ prox_status_t forward_kernels(prox_ffn* h, const void* x, int B, int k1, int k2,
   prox_status_t s;
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   h->sel_unordered = 0;
+  if (B > 1 && h->mask_policy == 1 && !(h->use_union && batch_path_ok(h, B, true))) return PROX_ERR_UNSUPPORTED;
   if (h->use_union && batch_path_ok(h, B, true)) {
     if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
     return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
@@ -790,6 +804,7 @@ prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x, int B, int k1, int 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = h->cfg.d_model;
   float* sc = scores ? scores : h->scores;
+  if (B > 1 && h->mask_policy == 1 && !(h->use_union && batch_path_ok(h, B, true))) return PROX_ERR_UNSUPPORTED;
   if (h->use_union && batch_path_ok(h, B, true)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st);
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, sc, st)) != PROX_OK) return s;
@@ -983,6 +998,12 @@ prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int
 prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on) {
   if (!h) return PROX_ERR_INVALID_ARG;
   h->use_fused = on != 0;
+  return PROX_OK;
+}
+
+prox_status_t prox_ffn_set_mask_policy(prox_ffn_t* h, int policy) {
+  if (!h || (policy != 0 && policy != 1)) return PROX_ERR_INVALID_ARG;
+  h->mask_policy = policy;
   return PROX_OK;
 }
 

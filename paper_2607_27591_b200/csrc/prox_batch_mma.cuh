@@ -724,13 +724,34 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
   }
 }
 
+// One mask for the whole batch (a policy beyond the paper): the channels are ranked by the sum of the
+// tokens' proxy scores, added token after token in fp32.
+__global__ void __launch_bounds__(256) shared_score_kernel(const float* __restrict__ scores, int B, int F,
+                                                           float* __restrict__ out) {
+  const int j = blockIdx.x * 256 + threadIdx.x;
+  if (j >= F) return;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += scores[(size_t)b * F + j];
+  out[j] = s;
+}
+
+// ... and every token's row of the mask output is that one list.
+__global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ sel, int sel_stride, int k2, int B) {
+  const int r = blockIdx.x * 256 + threadIdx.x;
+  if (r >= k2) return;
+  const int v = sel[r];
+  for (int b = 1; b < B; ++b) sel[(size_t)b * sel_stride + r] = v;
+}
+
 // Channel mask m_s of a token from its scores: exact top-k2 (ties: lower channel
 // first) by three radix steps over the score bits held in shared memory, then an
 // ordered list of the kept channels; the token's bit is also set in the channel's
 // byte of cmask (the union of the tokens' masks is read off those bytes).
+// token_bits = 0: block b is token b and sets bit b.  Otherwise (one shared mask for the batch: one block
+// over the summed scores) the kept channels get all of token_bits.
 __global__ void __launch_bounds__(kFusedThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
-                          unsigned* __restrict__ cmask) {
+                          unsigned* __restrict__ cmask, unsigned token_bits) {
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
   __shared__ unsigned hist[2048], wsum[32], wsum2[32];
@@ -793,7 +814,7 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
       if (gt || (eq && re < quota)) {
         const int ch = q * 4 + e;
         out[rg + min(re, quota)] = ch;
-        if (cmask) atomicOr(cmask + (ch >> 2), (1u << b) << (8 * (ch & 3)));
+        if (cmask) atomicOr(cmask + (ch >> 2), (token_bits ? token_bits : (1u << b)) << (8 * (ch & 3)));
       }
       rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
     }

@@ -753,6 +753,45 @@ def test_forms_on_odd_shapes(pb, D, F, bits, group):
         p.close()
 
 
+@pytest.mark.parametrize("group,B", [(0, 2), (128, 5), (128, 8)])
+def test_shared_batch_mask_policy(pb, toy, group, B):
+    """One channel mask for the batch, from the summed proxy scores; Stage 2 of every token on that mask."""
+    wl, p = toy
+    dg, du, _ = p.quantize(4, group)
+    k1, k2 = wl.points[50]
+    t0 = 4
+    pb.prox_ffn_set_mask_policy(p.h, 1)
+    try:
+        y = p.y_empty(B)
+        sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        used = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        xb = p.t_x[t0:t0 + B]
+        pb.prox_stage1_mask(p.h, xb, B, k1, k2, sel)
+        pb.prox_ffn_forward(p.h, xb, B, k1, k2, y)
+        pb.prox_ffn_last_mask(p.h, B, k2, used)
+        torch.cuda.synchronize()
+        sel_ref, thr, shared, _ = po.forward_batch_shared(p.x[t0:t0 + B], k1, k2, dg, du, p.wg, p.wu, p.wd)
+        sel_np, used_np, y_np = sel.cpu().numpy().astype(np.int64), used.cpu().numpy().astype(np.int64), y.cpu().numpy()
+        for b in range(B):
+            assert np.array_equal(sel_np[b], sel_np[0]) and np.array_equal(used_np[b], used_np[0])
+            check_mask(sel_np[b], shared, sel_ref, thr, k2, p.F)
+            check_mask(used_np[b], shared, sel_ref, thr, k2, p.F)
+            y_ref, _ = po.stage2(p.x[t0 + b], used_np[b], p.wg, p.wu, p.wd)
+            check_y(y_np[b], y_ref)
+        # one token: the policy changes nothing
+        _forward_check(pb, p, 2, k1, k2, B=1)
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        pb.prox_ffn_set_mask_policy(p.h, 0)
+    # 8-bit proxies do not have the tensor-core Stage 1: the policy is refused, not ignored
+    p.quantize(8, 0)
+    pb.prox_ffn_set_mask_policy(p.h, 1)
+    try:
+        assert pb.raw("prox_ffn_forward")(p.h, p.t_x[:2].data_ptr(), 2, k1, k2, p.y_empty(2).data_ptr(), None) == 2
+    finally:
+        pb.prox_ffn_set_mask_policy(p.h, 0)
+
+
 def test_pack_save_load_roundtrip(pb, toy, tmp_path):
     wl, p = toy
     p.quantize(4, 128)
