@@ -280,22 +280,16 @@ def ffn_stack(x_res, layers, eps: float, k1: int, k2: int):
 
 
 # ------------------------------------------------- a batch with one shared mask
-def forward_batch_shared(xs, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down, shared_inputs=False):
+def forward_batch_shared(xs, k1: int, k2: int, deq_gate, deq_up, w_gate, w_up, w_down):
     """A batch policy beyond the paper (it treats single-batch decoding only and
     names batching as future work): every token keeps its own input mask and
     its own proxy scores, the batch keeps ONE channel mask, the k2 channels of
     largest summed score  sum_b |s~_{b,j}|  (ties to the lower channel), and
     Stage 2 of every token runs on that mask.  With one token this is `forward`.
-    With `shared_inputs` the batch also keeps ONE input mask: the k1 inputs of
-    largest  max_b |x_{b,i}|  (ties to the lower index), used by every token's
-    proxy projections.
     Returns (sel, threshold, shared score, list of y per token)."""
     scores = []
-    idx_shared = None
-    if shared_inputs:
-        idx_shared = input_topk(np.max(np.abs(np.asarray(xs, dtype=np.float64)), axis=0), k1)
     for x in xs:
-        idx_x = idx_shared if shared_inputs else input_topk(x, k1)
+        idx_x = input_topk(x, k1)
         scores.append(proxy_scores(x, idx_x, deq_gate, deq_up))
     shared = np.zeros_like(scores[0])
     for sc in scores:                 # token after token

@@ -575,26 +575,3 @@ def test_shared_mask_batch_reduces_to_single_token_and_ignores_token_order():
         m[torch.from_numpy(sel3)] = 1.0
         np.testing.assert_allclose(ys3[b], (torch.from_numpy(wd) @ (s_full * m)).numpy(), rtol=1e-10, atol=1e-13)
         np.testing.assert_allclose(ysp[2 - b], ys3[b], rtol=0, atol=0)
-
-
-def test_shared_input_mask_of_a_batch():
-    wg, wu, wd, x = _problem(seed=32, n_tok=3)
-    dg = po.dequantize(*po.quantize_proxy(wg, 4, 0), 0)
-    du = po.dequantize(*po.quantize_proxy(wu, 4, 0), 0)
-    k1, k2 = 60, 80
-    # one token: nothing changes
-    one = po.forward(x[1], k1, k2, dg, du, wg, wu, wd)
-    sel, thr, _, ys = po.forward_batch_shared(x[1:2], k1, k2, dg, du, wg, wu, wd, shared_inputs=True)
-    assert np.array_equal(sel, one["sel"]) and np.array_equal(ys[0], one["y"])
-    # three tokens: the summed scores are those of the projections over the full-sort top-k1 of max_b |x|
-    sel3, _, shared3, _ = po.forward_batch_shared(x, k1, k2, dg, du, wg, wu, wd, shared_inputs=True)
-    m = np.max(np.abs(x), axis=0)
-    idx = np.sort(np.argsort(-m, kind="stable")[:k1])
-    ref = np.zeros(wg.shape[0])
-    for b in range(3):
-        xs = np.zeros_like(x[b]); xs[idx] = x[b][idx]
-        u = torch.from_numpy(du) @ torch.from_numpy(xs)
-        g = torch.from_numpy(dg) @ torch.from_numpy(xs)
-        ref += np.abs((u * torch.nn.functional.silu(g)).numpy())
-    np.testing.assert_allclose(shared3, ref, rtol=1e-11, atol=1e-14)
-    assert np.array_equal(sel3, np.sort(np.argsort(-shared3, kind="stable")[:k2]))
