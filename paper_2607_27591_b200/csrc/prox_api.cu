@@ -484,7 +484,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
 // ---- fused persistent kernel (batch 1) ----------------------------------------
 struct FusedPlan {
   bool ok;
-  int grid, ksplit, nstrips, big_bytes, nslots, xch;
+  int grid, pstages, big_bytes, nslots, xch;
   size_t smem;
   int optin;            // the device's opt-in limit: what the kernels' dynamic shared memory attribute is set to
 };
@@ -501,9 +501,11 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   pl.nslots = pl.big_bytes / (2 * D);
   if (pl.nslots > kMaxSlots) pl.nslots = kMaxSlots;
   if (pl.nslots < 3) return pl;
-  const int scb = 2 * ch_per_chunk(h->bits) * 2 * 32;                    // one (group, strip) scale block
-  if (pl.big_bytes < kFusedConsumerWarps * (kScaleGroupsPerWarp * scb + kProxyRowsInFlight * 512)) return pl;   // proxy row buffers
-  if (pl.big_bytes < kFusedConsumerWarps * 2 * ch_per_chunk(h->bits) * 32 * 4) return pl;      // reduction scratch
+  // the proxy GEMV keeps 16 tensor-memory columns per supergroup (4 scale groups), two sets of up to 256
+  if ((D / h->group + 3) / 4 > kMaxSuper) return pl;
+  pl.pstages = (pl.big_bytes - 1024) / kPStageBytes;
+  if (pl.pstages > kPStages) pl.pstages = kPStages;
+  if (pl.pstages < 4) return pl;
   if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
   if ((k2 + G - 1) / G + 2 > kMySelCap) return pl;       // a block's share: definite part + part of the threshold bin
   if (thresh) {
@@ -511,19 +513,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
     // must fit in shared memory (no radix fallback in this form), counts are kept in 16 bits
     if ((F + G - 1) / G + 2 > kMySelCap || (size_t)F * 4 + 256 > (size_t)pl.big_bytes || F >= 65536) return pl;
   }
-  pl.nstrips = nstrips_for(F, h->bits);
-  // row split: fill the grid evenly (items = strips * ksplit run in rounds of G blocks)
-  int best = 1;
-  double best_eff = -1.0;
-  const int ks_cap = k1 / 16 > 1 ? (k1 / 16 < 16 ? k1 / 16 : 16) : 1;
-  for (int ks = 1; ks <= ks_cap; ++ks) {
-    const int items = pl.nstrips * ks;
-    if ((size_t)items * 1024 > h->part_floats) break;
-    const int rounds = (items + G - 1) / G;
-    const double eff = (double)items / ((double)rounds * G);
-    if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
-  }
-  pl.ksplit = best;
+  (void)k1;
   pl.grid = G;
   pl.xch = D <= 4096 ? 4 : (D <= 8192 ? 2 : 1);          // warp groups of the down projection
   pl.smem = fixed + (size_t)pl.big_bytes;
@@ -585,8 +575,8 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.D = h->cfg.d_model; prm.F = h->cfg.d_ff; prm.k1 = k1; prm.k2 = k2;
   prm.gshift = (h->group == h->cfg.d_model) ? 31 : 7;
   prm.out_fp32 = h->cfg.out_dtype;
-  prm.nstrips = pl.nstrips; prm.ksplit = pl.ksplit;
-  prm.part = h->part; prm.ticket = h->ticket; prm.scores = h->scores; prm.ghist = h->syncbuf;
+  prm.pstages = pl.pstages;
+  prm.scores = h->scores; prm.ghist = h->syncbuf; prm.idx_out = h->idx_x;
   prm.sel_out = sel_out; prm.yacc = h->yacc;
   prm.bar_count = reinterpret_cast<unsigned long long*>(h->syncbuf + 2048); prm.done_ticket = h->syncbuf + 2050;
   prm.status = h->dev_status;
@@ -974,7 +964,7 @@ prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* inf
   CK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.optin));
   int nb = 0;
   CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kFusedThreads, pl.smem));
-  info[1] = pl.grid; info[2] = pl.ksplit; info[3] = (int)pl.smem; info[4] = pl.nslots;
+  info[1] = pl.grid; info[2] = pl.pstages; info[3] = (int)pl.smem; info[4] = pl.nslots;
   info[5] = fa.numRegs; info[6] = (int)fa.sharedSizeBytes; info[7] = nb;
   return PROX_OK;
 }

@@ -1,10 +1,12 @@
 // One persistent kernel for the whole batch-1 path (Sec. 4.1 Stage 1 + Stage 2):
 //
 //   A  every block: exact top-k1 of |x| (redundantly; x is a few KB)
-//   B  proxy GEMV over (channel strip, row split) items; the kept rows of the
-//      packed proxy land in shared memory through 16-byte async copies; split-K
-//      partials meet through a ticket counter; the last block of a strip writes
-//      the scores |u~ SiLU(g~)| and adds them to a global 2048-bin histogram
+//   B  proxy GEMV on the tensor cores (tcgen05, integer MMA, accumulators in
+//      tensor memory): a block owns 128-byte column tiles of the packed proxy
+//      over ALL kept rows, so the sums of a tile need no exchange with other
+//      blocks; the rows' bytes are the A operand as they lie in memory, x enters
+//      as signed base-256 digits; the block writes the scores |u~ SiLU(g~)| of
+//      its channels and adds them to a global 2048-bin histogram
 //   -- one grid-wide barrier (bounded spin, self-resetting) --
 //   C  every block (consumer warps only; the producer warps wait at the ring):
 //      the histogram gives the threshold bin b1; channels in bins above b1 are
@@ -28,6 +30,7 @@
 #pragma once
 
 #include "prox_kernels.cuh"
+#include "prox_umma.cuh"
 
 namespace prox {
 
@@ -44,8 +47,9 @@ constexpr int kChanBatch = 256;      // channels whose h values are held at once
 constexpr int kMySelCap = 512;       // channels one block may own
 constexpr int kCandCap = 4096;       // threshold-bin candidates kept in shared memory
 constexpr int kCand2Cap = 256;       // candidates left after the second refinement
-constexpr int kScaleGroupsPerWarp = 2;   // scale blocks a warp stages per item
-constexpr int kProxyRowsInFlight = 8;    // packed proxy rows a warp keeps in flight
+constexpr int kPStages = 16;             // ring of 32-row stages of the proxy GEMV (one per loader warp)
+constexpr int kPStageBytes = 9216;       // a stage: 4096 bytes of rows | 4096 low nibbles | 512 digits of x | pad
+constexpr int kMaxSuper = 16;            // supergroups (4 scale groups) whose accumulators fit the tensor memory
 constexpr unsigned kSpinLimit = 1u << 21;
 
 struct FusedParams {
@@ -53,8 +57,9 @@ struct FusedParams {
   const uint16_t* wg; const uint16_t* wu; const uint16_t* wdt;
   const uint16_t* x; void* y;
   int D, F, k1, k2, gshift, out_fp32;
-  int nstrips, ksplit;
-  float* part; unsigned* ticket; float* scores; unsigned* ghist; int* sel_out;
+  int pstages;        // stages of the proxy ring that fit (<= kPStages)
+  float* scores; unsigned* ghist; int* sel_out;
+  int* idx_out;       // the kept input list as this kernel built it (block 0 writes it; for checking)
   float* yacc; unsigned long long* bar_count; unsigned* done_ticket; int* status;
   int big_bytes;      // bytes of the large shared buffer
   int nslots;         // ring slots of D*2 bytes inside it
@@ -268,6 +273,14 @@ struct FusedSmem {
   int keys_s0, keys_s1;    // ring slots [s0, s1) that overlap the keys
   int list_s0, list_s1;    // ... and the list
   unsigned slot_use[kMaxSlots];   // uses of each ring slot whose data has been seen complete
+  unsigned long long pfull[kPStages];    // proxy ring: a stage is filled / has been read by the MMAs
+  unsigned long long pempty[kPStages];
+  unsigned long long acc_bar;            // all MMAs of a tile are complete
+  unsigned long long zero_bar;           // the accumulators are back at zero for the next tile
+  uint32_t tmem_base;
+  int sstart[kMaxSuper + 2];             // first kept row of every supergroup (and k1)
+  int bstart[kMaxSuper + 2];             // first 32-row block of every supergroup (and the block count)
+  float soff[4 * kMaxSuper];             // per scale group: code offset (8 or 128) * sum of the kept x, as integers
   float nsum[kFusedWarps][2];     // RMSNorm: the warps' sums of squares (hi, lo)
   float ninv[2];                  // ... and 1 / sqrt(mean + eps) (hi, lo)
 };
@@ -299,6 +312,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   if (tid < kMaxSlots) {
     mbar_init(smem_u32(&sm.mbar_full[tid]), 1);
     mbar_init(smem_u32(&sm.mbar_empty[tid]), kEmptyCount);
+    fence_mbar_init();
+  }
+  if (warp == 0) tmem_alloc_all(smem_u32(&sm.tmem_base));      // all 512 columns: one block per SM
+  if (tid < kPStages) {
+    mbar_init(smem_u32(&sm.pfull[tid]), 1);
+    mbar_init(smem_u32(&sm.pempty[tid]), 1);
+    if (tid == 0) { mbar_init(smem_u32(&sm.acc_bar), 1); mbar_init(smem_u32(&sm.zero_bar), kFusedConsumerWarps); }
     fence_mbar_init();
   }
   if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
@@ -360,7 +380,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     }
     for (int i = tid; i < 1024 + 32; i += NT) { if (i < 1024) sm.hist[i] = 0; else sm.hist2[i - 1024] = 0; }
   }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  if (warp < 4) {
+    // the accumulators of the proxy GEMV start at zero: 16 columns per supergroup, two sets 256 columns apart
+    const int ngz = (p.gshift >= 31) ? 1 : (D >> p.gshift);
+    const uint32_t tz = sm.tmem_base + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+    for (int c = 0; c < 16 * ((ngz + 3) >> 2); c += 16) { tmem_st16_zero(tz + (uint32_t)c); tmem_st16_zero(tz + 256u + (uint32_t)c); }
+    tmem_st_wait();
+    tc_fence_before();
+  }
   PROX_TRACE(1);
 
   // ------------------------------------------------- A: input mask (top-k1 of |x|)
@@ -444,187 +475,244 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     __syncthreads();
   }
 
+  if (cta == 0 && p.idx_out) {
+#pragma unroll 1
+    for (int i = tid; i < k1; i += NT) p.idx_out[i] = (int)idx16[i];
+  }
   PROX_TRACE(2);
-  // --------------------------------------- B: proxy GEMV, scores, score histogram
+  // --------------------------------------- B: proxy GEMV (tensor cores), scores, score histogram
+  // Per scale group g:  sum_k x_k q_kj = 2^(ebase-134) * sum_k X_k (byte_kj - offset), X_k the integer
+  // form of x_k (x_digits).  A block owns 128-byte tiles of the packed rows over all kept rows.  The kept
+  // rows are cut into blocks of at most 32 rows that stay inside one supergroup (4 scale groups); block b
+  // accumulates into 16 tensor-memory columns of its supergroup: column 4 * (g % 4) + d holds digit d of
+  // group g.  16 loader warps bring the rows in with plain 16-byte loads (8 in flight per lane) and store
+  // them (and the bytes with the high nibble masked off, and the digits of x) in a stage of the ring;
+  // one thread issues the MMAs; after the last one the 16 warps read the accumulators, apply the
+  // groups' scales and form the scores.
   {
+    constexpr bool LO = (BITS == 4);
     const int nchunks = F / CH;
-    const size_t row_bytes = (size_t)nchunks * 16;
-    const int nitems = p.nstrips * p.ksplit;
-    constexpr int SCB = NACC * 2 * 32;          // bytes of one (group, strip) scale block: 2 KB / 1 KB
-    constexpr int NBUF = kProxyRowsInFlight;    // 512-byte row buffers per warp, one async-copy group each
-    // per warp: [2 scale blocks][NBUF row buffers]
-    const uint32_t wscale = big_u32 + (uint32_t)warp * (uint32_t)(kScaleGroupsPerWarp * SCB + NBUF * 512);
-    const uint32_t wbuf = wscale + (uint32_t)(kScaleGroupsPerWarp * SCB);
-    for (int item = cta; item < nitems; item += G) {
-      const int strip = item % p.nstrips, ks = item / p.nstrips;
-      // 32-bit arithmetic on purpose (k1 <= 16384, ks < 64): a 64-bit division costs about a microsecond here
-      const int r0 = (int)(((unsigned)k1 * (unsigned)ks) / (unsigned)p.ksplit);
-      const int r1 = (int)(((unsigned)k1 * (unsigned)(ks + 1)) / (unsigned)p.ksplit);
-      float tot[NACC];
-#pragma unroll
-      for (int c = 0; c < NACC; ++c) tot[c] = 0.f;
+    const int row_bytes = nchunks * 16;
+    const int ntiles = (row_bytes + 127) >> 7;
+    const bool per_row = p.gshift >= 31;
+    const int ng = per_row ? 1 : (D >> p.gshift);
+    const int nsuper = (ng + 3) >> 2;
+    const int sgshift = per_row ? 31 : p.gshift + 2;
+    const uint32_t tbase = sm.tmem_base;
+    int* sd = reinterpret_cast<int*>(sm.hist2);               // [ng][4] digit sums of the kept x per group
+    // supergroup starts (lower bound in the ascending index list), largest exponent, digit sums
+    if (tid <= nsuper) {
+      int lo = 0, hi = k1;
+      if (tid == nsuper) lo = k1;
+      else {
+        const int lim = per_row ? 0 : (tid << sgshift);
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if ((int)idx16[mid] < lim) lo = mid + 1; else hi = mid; }
+      }
+      sm.sstart[tid] = lo;
+    }
+    unsigned mk = 0;
+    {
+      const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
+#pragma unroll 1
+      for (int i = tid; i < D / 2; i += NT) { const uint32_t w = xs32[i]; mk = max(mk, max(w & 0x7fffu, (w >> 16) & 0x7fffu)); }
+    }
+    mk = __reduce_max_sync(0xffffffffu, mk);
+    if (lane == 0) sm.wsum[warp] = mk;
+    if (tid < 4 * kMaxSuper * 4) sd[tid] = 0;
+    __syncthreads();
+    mk = __reduce_max_sync(0xffffffffu, lane < kFusedWarps ? sm.wsum[lane] : 0u);
+    const int emax = max((int)(mk >> 7), 1);
+    const int ebase = max(emax - 22, 1);
+    if (tid == 0) {
+      int acc = 0;
+      for (int s2 = 0; s2 < nsuper; ++s2) { sm.bstart[s2] = acc; acc += (sm.sstart[s2 + 1] - sm.sstart[s2] + 31) >> 5; }
+      sm.bstart[nsuper] = acc;
+    }
+#pragma unroll 1
+    for (int r = tid; r < k1; r += NT) {
+      const int i = idx16[r];
+      const uint32_t dg = x_digits(xs[i], ebase);
+      const int g = per_row ? 0 : (i >> p.gshift);
+      atomicAdd(&sd[g * 4 + 0], (int)(int8_t)(dg & 0xffu));
+      atomicAdd(&sd[g * 4 + 1], (int)(int8_t)((dg >> 8) & 0xffu));
+      atomicAdd(&sd[g * 4 + 2], (int)(int8_t)((dg >> 16) & 0xffu));
+      atomicAdd(&sd[g * 4 + 3], (int)(int8_t)(dg >> 24));
+    }
+    __syncthreads();
+    if (tid < ng)
+      sm.soff[tid] = (LO ? 8.f : 128.f) * digits_to_float((uint32_t)sd[tid * 4], (uint32_t)sd[tid * 4 + 1],
+                                                         (uint32_t)sd[tid * 4 + 2], (uint32_t)sd[tid * 4 + 3]);
+    const int nblk = sm.bstart[nsuper];
+    const int NSb = p.pstages;
+    const uint32_t ring = (big_u32 + 1023u) & ~1023u;
+    float* red = reinterpret_cast<float*>(sm.hist);           // [3][128][2] partial sums of warps 4..15
+    __syncthreads();
+    PROX_TRACE(29);
+    unsigned seq0 = 0;
+    int tile_iter = 0;
+    for (int tile = cta; tile < ntiles; tile += G, ++tile_iter) {
       if (warp < kFusedConsumerWarps) {
-        const int w0 = r0 + (int)(((unsigned)(r1 - r0) * (unsigned)warp) / (unsigned)kFusedConsumerWarps);
-        const int w1 = r0 + (int)(((unsigned)(r1 - r0) * (unsigned)(warp + 1)) / (unsigned)kFusedConsumerWarps);
-        const int nrows = w1 - w0;
-        const int seg = (int)min((size_t)512, row_bytes - (size_t)strip * 512);
-        const bool lane_valid = lane * 16 < seg;
-        const int chunk = strip * 32 + lane;
-        // Rows (and the scale blocks of the first two groups they touch) land in
-        // shared memory through 16-byte async copies, one copy group per row, so
-        // that a row can be consumed as soon as it is there.  Every lane later
-        // reads back exactly the bytes it copied itself: no barrier is needed.
-        const uint8_t* src0 = p.P + (size_t)strip * 512 + (size_t)lane * 16;
-        const int g_first = (nrows > 0) ? (idx16[w0] >> p.gshift) : 0;
-        const int g_last = (nrows > 0) ? (idx16[w1 - 1] >> p.gshift) : -1;
-        if (lane_valid) {
+        // ---- scales of this thread's byte column for the groups it will read back
+        const int q4 = warp & 3, part = warp >> 2;
+        const int col = q4 * 32 + lane;                        // byte column of the tile = data path lane
+        const int chunk = tile * 8 + (col >> 4);
+        const bool col_ok = chunk < nchunks;
+        uint32_t scl[16];
 #pragma unroll
-          for (int gq = 0; gq < kScaleGroupsPerWarp; ++gq) {
-            if (g_first + gq <= g_last) {
-              const uint8_t* ssrc = reinterpret_cast<const uint8_t*>(p.S + ((size_t)(g_first + gq) * nchunks + chunk) * NACC);
+        for (int it = 0; it < 4; ++it)
 #pragma unroll
-              for (int v4 = 0; v4 < NACC / 8; ++v4)
-                cp_async16(wscale + (uint32_t)(gq * SCB + lane * (NACC * 2) + v4 * 16), ssrc + v4 * 16);
+          for (int gq = 0; gq < 4; ++gq) {
+            const int g = 4 * (part + 4 * it) + gq;
+            uint32_t v = 0;
+            if (col_ok && g < ng) {
+              if (LO) v = __ldg(reinterpret_cast<const uint32_t*>(p.S + ((size_t)g * nchunks + chunk) * 32) + (col & 15));
+              else v = (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(p.S + ((size_t)g * nchunks + chunk) * 16) + (col & 15));
             }
+            scl[it * 4 + gq] = v;
           }
+        // ---- loader: blocks warp, warp + 16, ...
+#pragma unroll 1
+        for (int b = warp; b < nblk; b += kFusedConsumerWarps) {
+          int sg = 0;
+          while (sm.bstart[sg + 1] <= b) ++sg;
+          const int r0 = sm.sstart[sg] + ((b - sm.bstart[sg]) << 5);
+          const int nrows = min(32, sm.sstart[sg + 1] - r0);
+          const unsigned seq = seq0 + (unsigned)b;
+          const int st_i = (int)(seq % (unsigned)NSb);
+          const unsigned use = seq / (unsigned)NSb;
+          const int c = lane & 7, kq = lane >> 3;
+          const bool c_ok = tile * 8 + c < nchunks;
+          uint4 v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int kk = j * 4 + kq;
+            v[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (kk < nrows && c_ok)
+              v[j] = ld_stream(p.P + (size_t)idx16[r0 + kk] * (size_t)row_bytes + (size_t)tile * 128 + (size_t)c * 16);
+          }
+          uint4 brow = make_uint4(0u, 0u, 0u, 0u);
+          if (lane < nrows) {
+            const int i = idx16[r0 + lane];
+            const uint32_t dg = x_digits(xs[i], ebase);
+            const int slot = per_row ? 0 : ((i >> p.gshift) & 3);
+            brow.x = slot == 0 ? dg : 0u; brow.y = slot == 1 ? dg : 0u; brow.z = slot == 2 ? dg : 0u; brow.w = slot == 3 ? dg : 0u;
+          }
+          const bool free_ok = use == 0 || mbar_wait(smem_u32(&sm.pempty[st_i]), (use - 1u) & 1u, abortp);
+          if (!__all_sync(0xffffffffu, free_ok)) break;
+          const uint32_t stg = ring + (uint32_t)st_i * (uint32_t)kPStageBytes;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int kk = j * 4 + kq;
+            const uint32_t dst = stg + (uint32_t)((kk >> 3) * 1024 + (kk & 7) * 128 + ((c ^ (kk & 7)) << 4));
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v[j].x), "r"(v[j].y), "r"(v[j].z), "r"(v[j].w) : "memory");
+            if (LO)
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst + 4096u), "r"(v[j].x & 0x0f0f0f0fu), "r"(v[j].y & 0x0f0f0f0fu),
+                           "r"(v[j].z & 0x0f0f0f0fu), "r"(v[j].w & 0x0f0f0f0fu) : "memory");
+          }
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + 8192u + (uint32_t)lane * 16u), "r"(brow.x), "r"(brow.y), "r"(brow.z), "r"(brow.w) : "memory");
+          fence_proxy_async();                 // the tensor core reads the stage through the async proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive_n(smem_u32(&sm.pfull[st_i]), 1u);
         }
-        cp_async_commit();
-        auto issue_row = [&](int rr) {                    // always commits, so group counting stays uniform
-          if (rr < nrows && lane_valid) {
-            const int i = idx16[w0 + rr];
-            cp_async16(wbuf + (uint32_t)(rr % NBUF) * 512u + (uint32_t)lane * 16u, src0 + (size_t)i * row_bytes);
-          }
-          cp_async_commit();
-        };
+        // ---- read the accumulators back: thread = byte column, warp part p takes supergroups p, p + 4, ...
+        const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u, abortp));
+        tc_fence_after();
+        float t0 = 0.f, t1 = 0.f;              // 4-bit: sums of the low / high nibble's channel; 8-bit: t0 only
+        const bool more = tile + G < ntiles;
 #pragma unroll
-        for (int rr = 0; rr < NBUF; ++rr) issue_row(rr);
-        PROX_TRACE(29);
-        float acc[NACC];
+        for (int it = 0; it < 4; ++it) {
+          const int sg = part + 4 * it;
+          if (sg < nsuper && acc_ok) {         // warp-uniform
+            uint32_t a[16], l[16];
+            const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(16 * sg);
+            tmem_ld16(ta, a);
+            if (LO) tmem_ld16(ta + 256u, l);
+            tmem_ld_wait();
+            if (more) { tmem_st16_zero(ta); if (LO) tmem_st16_zero(ta + 256u); }
 #pragma unroll
-        for (int c = 0; c < NACC; ++c) acc[c] = 0.f;
-        int curg = -1;
-        auto flush = [&](int g) {
-          if (g < 0 || !lane_valid) return;
-          uint4 sv[NACC / 8];
-          if (g - g_first < kScaleGroupsPerWarp) {
-#pragma unroll
-            for (int v4 = 0; v4 < NACC / 8; ++v4)
-              sv[v4] = lds128(wscale + (uint32_t)((g - g_first) * SCB + lane * (NACC * 2) + v4 * 16));
-          } else {
-            const uint4* sp = reinterpret_cast<const uint4*>(p.S + ((size_t)g * nchunks + chunk) * NACC);
-#pragma unroll
-            for (int v4 = 0; v4 < NACC / 8; ++v4) sv[v4] = __ldg(sp + v4);
-          }
-#pragma unroll
-          for (int v4 = 0; v4 < NACC / 8; ++v4) {
-            const uint32_t sw[4] = {sv[v4].x, sv[v4].y, sv[v4].z, sv[v4].w};
-#pragma unroll
-            for (int h2 = 0; h2 < 4; ++h2) {
-              const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&sw[h2]));
-              const int c = v4 * 8 + h2 * 2;
-              tot[c] = fmaf(sc.x, acc[c], tot[c]);
-              tot[c + 1] = fmaf(sc.y, acc[c + 1], tot[c + 1]);
-              acc[c] = 0.f; acc[c + 1] = 0.f;
-            }
-          }
-        };
-        for (int rr = 0; rr < nrows; ++rr) {
-          cp_async_wait<NBUF - 1>();                      // the group of row rr (and the scales) has landed
-          if (rr == 0) PROX_TRACE(27);
-          const int i = idx16[w0 + rr];
-          const float xv = xf[i];
-          const int g = i >> p.gshift;
-          if (g != curg) { flush(curg); curg = g; }
-          if (lane_valid) {
-            const uint4 v = lds128(wbuf + (uint32_t)(rr % NBUF) * 512u + (uint32_t)lane * 16u);
-            proxy_accumulate_exact<BITS>(v, xv, acc);
-          }
-          issue_row(rr + NBUF);
-        }
-        cp_async_wait<0>();
-        flush(curg);
-      }
-      PROX_TRACE(22);
-      __syncthreads();                         // every warp is done with its row buffers
-      PROX_TRACE(23);
-      float* red = reinterpret_cast<float*>(big);
-      if (warp < kFusedConsumerWarps) {
-#pragma unroll
-        for (int c = 0; c < NACC; ++c) red[warp * (NACC * 32) + c * 32 + lane] = tot[c];
-      }
-      __syncthreads();
-      constexpr int NV = NACC * 32;            // values per strip: 1024 (4-bit) or 512 (8-bit)
-      float sumv[2] = {0.f, 0.f};
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const int k = tid + q * NT;
-        if (k < NV) {
-          float s = 0.f;
-#pragma unroll
-          for (int w = 0; w < kFusedConsumerWarps; ++w) s += red[w * NV + k];
-          sumv[q] = s;
-        }
-      }
-      __syncthreads();
-      PROX_TRACE(24);
-      float* fin = red;
-      bool last = true;
-      if (p.ksplit > 1) {
-        float* pb = p.part + ((size_t)ks * p.nstrips + strip) * NV;
-#pragma unroll
-        for (int q = 0; q < 2; ++q) { const int k = tid + q * NT; if (k < NV) __stcg(pb + k, sumv[q]); }
-        __syncthreads();
-        if (tid == 0) {
-          __threadfence();                      // publishes the whole block's partials (seen through the barrier)
-          const unsigned tk = atomicAdd(&p.ticket[strip], 1u);
-          sm.s_last = (tk == (unsigned)(p.ksplit - 1));
-          __threadfence();
-        }
-        __syncthreads();
-        last = sm.s_last != 0;
-        PROX_TRACE(25);
-        if (last) {
-          float s4[2] = {0.f, 0.f};
-          for (int z0 = 0; z0 < p.ksplit; z0 += 8) {         // loads of a batch are independent
-            float t[8][2];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const float* pz = p.part + ((size_t)(z0 + u) * p.nstrips + strip) * NV;
-#pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                const int k = tid + q * NT;
-                t[u][q] = (z0 + u < p.ksplit && k < NV) ? __ldcg(pz + k) : 0.f;
+            for (int gq = 0; gq < 4; ++gq) {
+              const int g = 4 * sg + gq;
+              if (g < ng) {
+                const float off = sm.soff[g];
+                const float fa = digits_to_float(a[4 * gq], a[4 * gq + 1], a[4 * gq + 2], a[4 * gq + 3]);
+                if (LO) {
+                  const float fl = digits_to_float(l[4 * gq], l[4 * gq + 1], l[4 * gq + 2], l[4 * gq + 3]);
+                  const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&scl[it * 4 + gq]));
+                  t0 = fmaf(sc.x, fl - off, t0);
+                  t1 = fmaf(sc.y, fmaf(fa - fl, 0.0625f, -off), t1);
+                } else {
+                  const float sc = __half2float(__ushort_as_half((unsigned short)scl[it * 4 + gq]));
+                  t0 = fmaf(sc, fa - off, t0);
+                }
               }
             }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) { s4[0] += t[u][0]; s4[1] += t[u][1]; }
-          }
-#pragma unroll
-          for (int q = 0; q < 2; ++q) { const int k = tid + q * NT; if (k < NV) fin[k] = s4[q]; }
-          if (tid == 0) p.ticket[strip] = 0;
-        }
-      } else {
-#pragma unroll
-        for (int q = 0; q < 2; ++q) { const int k = tid + q * NT; if (k < NV) fin[k] = sumv[q]; }
-      }
-      PROX_TRACE(26);
-      if (last) {
-        for (int i = tid; i < 2048; i += NT) sm.hist[i] = 0;
-        __syncthreads();
-        for (int k = tid; k < CH * 32; k += NT) {
-          const int c = k >> 5, ln = k & 31;
-          const int ch = (strip * 32 + ln) * CH + c;
-          if (ch < F) {
-            const float sc = fabsf(fin[k + CH * 32] * silu_fast(fin[k]));
-            __stcg(p.scores + ch, sc);
-            atomicAdd(&sm.hist[__float_as_uint(sc) >> 20], 1u);
           }
         }
-        __syncthreads();
-        for (int i = tid; i < 2048; i += NT) { const unsigned v = sm.hist[i]; if (v) atomicAdd(p.ghist + i, v); }
+        if (more) { tmem_st_wait(); tc_fence_before(); }
+        if (part > 0) { red[((part - 1) * 128 + col) * 2] = t0; red[((part - 1) * 128 + col) * 2 + 1] = t1; }
+        consumer_sync();
+        if (more && lane == 0) mbar_arrive_n(smem_u32(&sm.zero_bar), 1u);
+        if (part == 0) {
+#pragma unroll
+          for (int pp = 0; pp < 3; ++pp) { t0 += red[(pp * 128 + col) * 2]; t1 += red[(pp * 128 + col) * 2 + 1]; }
+          t0 = scalbnf(t0, ebase - 134); t1 = scalbnf(t1, ebase - 134);
+          // bytes 0..7 of a chunk hold gate codes, bytes 8..15 the up codes of the same channels
+          const float u0 = __shfl_xor_sync(0xffffffffu, t0, 8), u1 = __shfl_xor_sync(0xffffffffu, t1, 8);
+          if ((col & 8) == 0 && col_ok) {
+            if (LO) {
+              const int ch = chunk * 16 + 2 * (col & 7);
+              const float s0 = fabsf(u0 * silu_fast(t0)), s1 = fabsf(u1 * silu_fast(t1));
+              __stcg(reinterpret_cast<float2*>(p.scores + ch), make_float2(s0, s1));
+              atomicAdd(p.ghist + (__float_as_uint(s0) >> 20), 1u);
+              atomicAdd(p.ghist + (__float_as_uint(s1) >> 20), 1u);
+            } else {
+              const int ch = chunk * 8 + (col & 7);
+              const float s0 = fabsf(u0 * silu_fast(t0));
+              __stcg(p.scores + ch, s0);
+              atomicAdd(p.ghist + (__float_as_uint(s0) >> 20), 1u);
+            }
+          }
+        }
+        consumer_sync();                       // red is free again
+      } else if (warp == kFusedConsumerWarps) {
+        // ---- one thread issues the MMAs, block by block
+        if (lane == 0) {
+          bool ok = true;
+          if (tile_iter > 0) ok = mbar_wait(smem_u32(&sm.zero_bar), (unsigned)(tile_iter - 1) & 1u, abortp);
+          tc_fence_after();
+          constexpr uint32_t idesc = umma_idesc_u8s8(128, 16);
+          int sg = 0;
+#pragma unroll 1
+          for (int b = 0; b < nblk && ok; ++b) {
+            while (sm.bstart[sg + 1] <= b) ++sg;
+            const unsigned seq = seq0 + (unsigned)b;
+            const int st_i = (int)(seq % (unsigned)NSb);
+            const unsigned use = seq / (unsigned)NSb;
+            ok = mbar_wait(smem_u32(&sm.pfull[st_i]), use & 1u, abortp);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t stg = ring + (uint32_t)st_i * (uint32_t)kPStageBytes;
+            const uint64_t bdesc = umma_smem_desc(stg + 8192u, 128u, 512u, 0u);
+            umma_i8(tbase + (uint32_t)(16 * sg), umma_smem_desc(stg, 4096u, 1024u, 2u), bdesc, idesc, 1u);
+            if (LO) umma_i8(tbase + 256u + (uint32_t)(16 * sg), umma_smem_desc(stg + 4096u, 4096u, 1024u, 2u), bdesc, idesc, 1u);
+            umma_commit(smem_u32(&sm.pempty[st_i]));
+          }
+          umma_commit(smem_u32(&sm.acc_bar));
+          if (!ok) {                               // nothing may be in flight when the block frees the tensor memory
+#pragma unroll 1
+            for (unsigned it = 0; it < 65536u; ++it) {
+              if (mbar_try_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u)) break;
+              __nanosleep(64);
+            }
+          }
+        }
       }
-      __syncthreads();
+      seq0 += (unsigned)nblk;
     }
+    // the tensor memory is not used after this phase
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_free_all(tbase);
   }
 
   PROX_TRACE(3);
