@@ -505,7 +505,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   if ((D / h->group + 3) / 4 > kMaxSuper) return pl;
   pl.pstages = (pl.big_bytes - 1024) / kPStageBytes;
   if (pl.pstages > kPStages) pl.pstages = kPStages;
-  if (pl.pstages < 4) return pl;
+  if (pl.pstages < kPStages) return pl;                                   // every loader warp owns a stage
   if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
   if ((k2 + G - 1) / G + 2 > kMySelCap) return pl;       // a block's share: definite part + part of the threshold bin
   if (thresh) {

@@ -134,6 +134,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 #define PROX_TRACE_AT(k, who) do { if (p.trace && tid == (who)) p.trace[(size_t)cta * 32 + (k)] = global_ns(); } while (0)
 #define PROX_TRACE(k) do { if (p.trace && tid == 0) p.trace[(size_t)cta * 32 + (k)] = global_ns(); } while (0)
+__device__ __forceinline__ bool elect_one() {          // the same lane every time for a full warp
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P1;\n\telect.sync _|P1, 0xffffffff;\n\tselp.u32 %0, 1, 0, P1;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void settler_sync() {      // the lower half of the consumer warps
   asm volatile("bar.sync 3, %0;" ::"n"(kSettlers) : "memory");
 }
@@ -273,10 +278,8 @@ struct FusedSmem {
   int keys_s0, keys_s1;    // ring slots [s0, s1) that overlap the keys
   int list_s0, list_s1;    // ... and the list
   unsigned slot_use[kMaxSlots];   // uses of each ring slot whose data has been seen complete
-  unsigned long long pfull[kPStages];    // proxy ring: a stage is filled / has been read by the MMAs
-  unsigned long long pempty[kPStages];
-  unsigned long long acc_bar;            // all MMAs of a tile are complete
-  unsigned long long zero_bar;           // the accumulators are back at zero for the next tile
+  unsigned long long pempty[kPStages];   // proxy ring: the MMAs have read the stage of warp w
+  unsigned long long acc_bar;            // all MMAs of a tile are complete (one arrival per loader warp)
   uint32_t tmem_base;
   int sstart[kMaxSuper + 2];             // first kept row of every supergroup (and k1)
   int bstart[kMaxSuper + 2];             // first 32-row block of every supergroup (and the block count)
@@ -316,9 +319,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   }
   if (warp == 0) tmem_alloc_all(smem_u32(&sm.tmem_base));      // all 512 columns: one block per SM
   if (tid < kPStages) {
-    mbar_init(smem_u32(&sm.pfull[tid]), 1);
     mbar_init(smem_u32(&sm.pempty[tid]), 1);
-    if (tid == 0) { mbar_init(smem_u32(&sm.acc_bar), 1); mbar_init(smem_u32(&sm.zero_bar), kFusedConsumerWarps); }
+    if (tid == 0) mbar_init(smem_u32(&sm.acc_bar), kFusedConsumerWarps);
     fence_mbar_init();
   }
   if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
@@ -499,16 +501,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     const int nsuper = (ng + 3) >> 2;
     const int sgshift = per_row ? 31 : p.gshift + 2;
     const uint32_t tbase = sm.tmem_base;
-    int* sd = reinterpret_cast<int*>(sm.hist2);               // [ng][4] digit sums of the kept x per group
-    // supergroup starts (lower bound in the ascending index list), largest exponent, digit sums
-    if (tid <= nsuper) {
+    int* gstart = reinterpret_cast<int*>(sm.hist2);           // [ng + 1] first kept row of every scale group (and k1)
+    // group starts (lower bound in the ascending index list) and the largest exponent
+    if (tid <= ng) {
       int lo = 0, hi = k1;
-      if (tid == nsuper) lo = k1;
+      if (tid == ng) lo = k1;
       else {
-        const int lim = per_row ? 0 : (tid << sgshift);
+        const int lim = per_row ? 0 : (tid << p.gshift);
         while (lo < hi) { const int mid = (lo + hi) >> 1; if ((int)idx16[mid] < lim) lo = mid + 1; else hi = mid; }
       }
-      sm.sstart[tid] = lo;
+      gstart[tid] = lo;
     }
     unsigned mk = 0;
     {
@@ -518,43 +520,55 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     }
     mk = __reduce_max_sync(0xffffffffu, mk);
     if (lane == 0) sm.wsum[warp] = mk;
-    if (tid < 4 * kMaxSuper * 4) sd[tid] = 0;
     __syncthreads();
     mk = __reduce_max_sync(0xffffffffu, lane < kFusedWarps ? sm.wsum[lane] : 0u);
     const int emax = max((int)(mk >> 7), 1);
     const int ebase = max(emax - 22, 1);
     if (tid == 0) {
       int acc = 0;
-      for (int s2 = 0; s2 < nsuper; ++s2) { sm.bstart[s2] = acc; acc += (sm.sstart[s2 + 1] - sm.sstart[s2] + 31) >> 5; }
+      for (int s2 = 0; s2 <= nsuper; ++s2) {
+        const int r = gstart[min(4 * s2, ng)];
+        sm.sstart[s2] = r;
+        if (s2 > 0) { sm.bstart[s2 - 1] = acc; acc += (r - sm.sstart[s2 - 1] + 31) >> 5; }
+      }
       sm.bstart[nsuper] = acc;
     }
+    // per scale group: offset * sum of the kept x as integers (a warp per group, no atomics)
 #pragma unroll 1
-    for (int r = tid; r < k1; r += NT) {
-      const int i = idx16[r];
-      const uint32_t dg = x_digits(xs[i], ebase);
-      const int g = per_row ? 0 : (i >> p.gshift);
-      atomicAdd(&sd[g * 4 + 0], (int)(int8_t)(dg & 0xffu));
-      atomicAdd(&sd[g * 4 + 1], (int)(int8_t)((dg >> 8) & 0xffu));
-      atomicAdd(&sd[g * 4 + 2], (int)(int8_t)((dg >> 16) & 0xffu));
-      atomicAdd(&sd[g * 4 + 3], (int)(int8_t)(dg >> 24));
+    for (int g = warp; g < ng; g += kFusedWarps) {
+      int d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+#pragma unroll 1
+      for (int r = gstart[g] + lane; r < gstart[g + 1]; r += 32) {
+        const uint32_t dg = x_digits(xs[idx16[r]], ebase);
+        d0 += (int)(int8_t)(dg & 0xffu); d1 += (int)(int8_t)((dg >> 8) & 0xffu);
+        d2 += (int)(int8_t)((dg >> 16) & 0xffu); d3 += (int)(int8_t)(dg >> 24);
+      }
+      d0 = __reduce_add_sync(0xffffffffu, d0); d1 = __reduce_add_sync(0xffffffffu, d1);
+      d2 = __reduce_add_sync(0xffffffffu, d2); d3 = __reduce_add_sync(0xffffffffu, d3);
+      if (lane == 0) sm.soff[g] = (LO ? 8.f : 128.f) * digits_to_float((uint32_t)d0, (uint32_t)d1, (uint32_t)d2, (uint32_t)d3);
     }
     __syncthreads();
-    if (tid < ng)
-      sm.soff[tid] = (LO ? 8.f : 128.f) * digits_to_float((uint32_t)sd[tid * 4], (uint32_t)sd[tid * 4 + 1],
-                                                         (uint32_t)sd[tid * 4 + 2], (uint32_t)sd[tid * 4 + 3]);
     const int nblk = sm.bstart[nsuper];
-    const int NSb = p.pstages;
     const uint32_t ring = (big_u32 + 1023u) & ~1023u;
     float* red = reinterpret_cast<float*>(sm.hist);           // [3][128][2] partial sums of warps 4..15
-    __syncthreads();
     PROX_TRACE(29);
-    unsigned seq0 = 0;
-    int tile_iter = 0;
-    for (int tile = cta; tile < ntiles; tile += G, ++tile_iter) {
-      if (warp < kFusedConsumerWarps) {
+    if (warp < kFusedConsumerWarps) {
+      // a warp owns one stage of the ring: it fills it and issues the stage's MMAs itself (the tensor core
+      // takes accumulating MMAs from several threads into the same columns; integer sums do not depend on the order)
+      const uint32_t stg = ring + (uint32_t)warp * (uint32_t)kPStageBytes;
+      const uint64_t adesc = umma_smem_desc(stg, 4096u, 1024u, 2u);
+      const uint64_t ldesc = umma_smem_desc(stg + 4096u, 4096u, 1024u, 2u);
+      const uint64_t bdesc = umma_smem_desc(stg + 8192u, 128u, 512u, 0u);
+      constexpr uint32_t idesc = umma_idesc_u8s8(128, 16);
+      const uint32_t my_empty = smem_u32(&sm.pempty[warp]);
+      const int q4 = warp & 3, part = warp >> 2;
+      const int col = q4 * 32 + lane;                          // byte column of the tile = data path lane
+      const int c = lane & 7, kq = lane >> 3;
+      unsigned uses = 0;                                       // stages this warp has handed to the tensor core
+      int tile_iter = 0;
+#pragma unroll 1
+      for (int tile = cta; tile < ntiles; tile += G, ++tile_iter) {
         // ---- scales of this thread's byte column for the groups it will read back
-        const int q4 = warp & 3, part = warp >> 2;
-        const int col = q4 * 32 + lane;                        // byte column of the tile = data path lane
         const int chunk = tile * 8 + (col >> 4);
         const bool col_ok = chunk < nchunks;
         uint32_t scl[16];
@@ -570,18 +584,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             }
             scl[it * 4 + gq] = v;
           }
-        // ---- loader: blocks warp, warp + 16, ...
+        const bool c_ok = tile * 8 + c < nchunks;
+        bool alive_b = true;
+        int sg = 0;
 #pragma unroll 1
         for (int b = warp; b < nblk; b += kFusedConsumerWarps) {
-          int sg = 0;
           while (sm.bstart[sg + 1] <= b) ++sg;
           const int r0 = sm.sstart[sg] + ((b - sm.bstart[sg]) << 5);
           const int nrows = min(32, sm.sstart[sg + 1] - r0);
-          const unsigned seq = seq0 + (unsigned)b;
-          const int st_i = (int)(seq % (unsigned)NSb);
-          const unsigned use = seq / (unsigned)NSb;
-          const int c = lane & 7, kq = lane >> 3;
-          const bool c_ok = tile * 8 + c < nchunks;
           uint4 v[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -590,6 +600,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             if (kk < nrows && c_ok)
               v[j] = ld_stream(p.P + (size_t)idx16[r0 + kk] * (size_t)row_bytes + (size_t)tile * 128 + (size_t)c * 16);
           }
+          if (b == 0) PROX_TRACE(22);
           uint4 brow = make_uint4(0u, 0u, 0u, 0u);
           if (lane < nrows) {
             const int i = idx16[r0 + lane];
@@ -597,9 +608,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             const int slot = per_row ? 0 : ((i >> p.gshift) & 3);
             brow.x = slot == 0 ? dg : 0u; brow.y = slot == 1 ? dg : 0u; brow.z = slot == 2 ? dg : 0u; brow.w = slot == 3 ? dg : 0u;
           }
-          const bool free_ok = use == 0 || mbar_wait(smem_u32(&sm.pempty[st_i]), (use - 1u) & 1u, abortp);
-          if (!__all_sync(0xffffffffu, free_ok)) break;
-          const uint32_t stg = ring + (uint32_t)st_i * (uint32_t)kPStageBytes;
+          const bool free_ok = uses == 0 || mbar_wait(my_empty, (uses - 1u) & 1u, abortp);
+          if (!__all_sync(0xffffffffu, free_ok)) { alive_b = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int kk = j * 4 + kq;
@@ -612,26 +622,37 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + 8192u + (uint32_t)lane * 16u), "r"(brow.x), "r"(brow.y), "r"(brow.z), "r"(brow.w) : "memory");
           fence_proxy_async();                 // the tensor core reads the stage through the async proxy
           __syncwarp();
-          if (lane == 0) mbar_arrive_n(smem_u32(&sm.pfull[st_i]), 1u);
+          if (elect_one()) {
+            umma_i8(tbase + (uint32_t)(16 * sg), adesc, bdesc, idesc, 1u);
+            if (LO) umma_i8(tbase + 256u + (uint32_t)(16 * sg), ldesc, bdesc, idesc, 1u);
+            umma_commit(my_empty);
+          }
+          __syncwarp();
+          ++uses;
+          if (b == 0) PROX_TRACE(23);
         }
+        if (elect_one()) umma_commit(smem_u32(&sm.acc_bar));   // one arrival per warp once its MMAs are complete
+        __syncwarp();
+        PROX_TRACE(24);
         // ---- read the accumulators back: thread = byte column, warp part p takes supergroups p, p + 4, ...
-        const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u, abortp));
+        const bool acc_ok = __all_sync(0xffffffffu, alive_b && mbar_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u, abortp));
         tc_fence_after();
+        PROX_TRACE(25);
         float t0 = 0.f, t1 = 0.f;              // 4-bit: sums of the low / high nibble's channel; 8-bit: t0 only
         const bool more = tile + G < ntiles;
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
-          const int sg = part + 4 * it;
-          if (sg < nsuper && acc_ok) {         // warp-uniform
+          const int sgd = part + 4 * it;
+          if (sgd < nsuper && acc_ok) {        // warp-uniform
             uint32_t a[16], l[16];
-            const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(16 * sg);
+            const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(16 * sgd);
             tmem_ld16(ta, a);
             if (LO) tmem_ld16(ta + 256u, l);
             tmem_ld_wait();
             if (more) { tmem_st16_zero(ta); if (LO) tmem_st16_zero(ta + 256u); }
 #pragma unroll
             for (int gq = 0; gq < 4; ++gq) {
-              const int g = 4 * sg + gq;
+              const int g = 4 * sgd + gq;
               if (g < ng) {
                 const float off = sm.soff[g];
                 const float fa = digits_to_float(a[4 * gq], a[4 * gq + 1], a[4 * gq + 2], a[4 * gq + 3]);
@@ -648,10 +669,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             }
           }
         }
+        PROX_TRACE(26);
         if (more) { tmem_st_wait(); tc_fence_before(); }
         if (part > 0) { red[((part - 1) * 128 + col) * 2] = t0; red[((part - 1) * 128 + col) * 2 + 1] = t1; }
         consumer_sync();
-        if (more && lane == 0) mbar_arrive_n(smem_u32(&sm.zero_bar), 1u);
+        if (more) tc_fence_after();            // every warp's columns are back at zero before the next tile's MMAs
         if (part == 0) {
 #pragma unroll
           for (int pp = 0; pp < 3; ++pp) { t0 += red[(pp * 128 + col) * 2]; t1 += red[(pp * 128 + col) * 2 + 1]; }
@@ -673,41 +695,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             }
           }
         }
-        consumer_sync();                       // red is free again
-      } else if (warp == kFusedConsumerWarps) {
-        // ---- one thread issues the MMAs, block by block
-        if (lane == 0) {
-          bool ok = true;
-          if (tile_iter > 0) ok = mbar_wait(smem_u32(&sm.zero_bar), (unsigned)(tile_iter - 1) & 1u, abortp);
-          tc_fence_after();
-          constexpr uint32_t idesc = umma_idesc_u8s8(128, 16);
-          int sg = 0;
+        if (more) consumer_sync();             // red is free again
+      }
+      // nothing may be in flight when the block frees the tensor memory (only a block whose wait expired gets here early)
+      if (sm.abort_flag && lane == 0) {
 #pragma unroll 1
-          for (int b = 0; b < nblk && ok; ++b) {
-            while (sm.bstart[sg + 1] <= b) ++sg;
-            const unsigned seq = seq0 + (unsigned)b;
-            const int st_i = (int)(seq % (unsigned)NSb);
-            const unsigned use = seq / (unsigned)NSb;
-            ok = mbar_wait(smem_u32(&sm.pfull[st_i]), use & 1u, abortp);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t stg = ring + (uint32_t)st_i * (uint32_t)kPStageBytes;
-            const uint64_t bdesc = umma_smem_desc(stg + 8192u, 128u, 512u, 0u);
-            umma_i8(tbase + (uint32_t)(16 * sg), umma_smem_desc(stg, 4096u, 1024u, 2u), bdesc, idesc, 1u);
-            if (LO) umma_i8(tbase + 256u + (uint32_t)(16 * sg), umma_smem_desc(stg + 4096u, 4096u, 1024u, 2u), bdesc, idesc, 1u);
-            umma_commit(smem_u32(&sm.pempty[st_i]));
-          }
-          umma_commit(smem_u32(&sm.acc_bar));
-          if (!ok) {                               // nothing may be in flight when the block frees the tensor memory
-#pragma unroll 1
-            for (unsigned it = 0; it < 65536u; ++it) {
-              if (mbar_try_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u)) break;
-              __nanosleep(64);
-            }
-          }
+        for (unsigned it = 0; it < 65536u && uses > 0; ++it) {
+          if (mbar_try_wait(my_empty, (uses - 1u) & 1u)) break;
+          __nanosleep(64);
         }
       }
-      seq0 += (unsigned)nblk;
     }
     // the tensor memory is not used after this phase
     tc_fence_before();
