@@ -128,8 +128,8 @@ prox_status_t prox_ffn_forward(prox_ffn_t* h, const void* x_dev, int B, int k1, 
  * (cooperative launch, one block per SM, one grid-wide barrier with a bounded
  * wait between Stage 1 and Stage 2); prox_ffn_set_fused(h, 0) selects the
  * kernel-per-step path instead (always used for B > 1).  If a bounded wait
- * ever expires the kernel leaves, y is not written and
- * prox_last_device_status reports bit 4. */
+ * ever expires the kernel leaves, y is not written (undefined) and
+ * prox_last_device_status reports bit 4 and returns PROX_ERR_TIMEOUT. */
 prox_status_t prox_ffn_set_fused(prox_ffn_t* h, int on);
 
 /* Mask policy of calls with B > 1 (the paper treats batch 1 only and names batching as future work):
@@ -170,6 +170,19 @@ prox_status_t prox_fused_kernel_info(prox_ffn_t* h, int k1, int k2, int32_t* inf
  * copied to it as [min(max_blocks, SM count)][32] uint64 (synchronises).
  * on = 0 frees the buffer. */
 prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int max_blocks);
+
+/* Test hook: what Stage 1 of the most recent forward call at B = 1 itself computed: its kept-input
+ * list (first indicator of Sec. 4.1; dev int32 [k1], ascending; NULL to skip) and its proxy scores
+ * (|u~ SiLU(g~)|, dev fp32 [d_ff]; NULL to skip).  Enqueued on stream. */
+prox_status_t prox_ffn_last_stage1(prox_ffn_t* h, int k1, int32_t* idx_dev_or_null, float* scores_dev_or_null,
+                                   void* stream);
+
+/* Test hook for the bounded device-side waits: spin_limit = polls after which a wait gives up
+ * (0 = the default, about two million); barrier_bias > 0 keeps the grid barrier of the persistent
+ * kernel from ever completing, so that the next B = 1 forward call runs into the limit, leaves
+ * without writing y and reports it (see prox_last_device_status).  Nothing hangs or faults: the
+ * blocks give up and return.  Set both back to 0 afterwards. */
+prox_status_t prox_debug_set_wait(prox_ffn_t* h, uint32_t spin_limit, uint32_t barrier_bias);
 
 /* Copy the channel mask of the most recent prox_ffn_forward call (top-k rule)
  * into sel_dev, dev int32 [B, k2], ascending per token.  Enqueued on stream. */
@@ -329,7 +342,12 @@ prox_status_t prox_algorithmic_bytes(const prox_ffn_t* h, int rows_in, int rows_
 /* Device-side diagnostics: 0 if no kernel recorded a problem since the last
  * read; otherwise a bit set (1 = channel id out of range skipped, 2 = input id
  * out of range skipped, 4 = bounded wait expired).  Reading clears it.
- * Synchronises the given stream. */
+ * Synchronises the given stream.  If bit 4 is set the call that ran into the wait
+ * did not write its output (y is undefined); the handle's shared counters are put
+ * back to their idle state here and the call returns PROX_ERR_TIMEOUT (with *code
+ * filled in); the next forward call is an ordinary one.  prox_ffn_forward_host,
+ * which synchronises anyway, checks for an expired wait itself and returns
+ * PROX_ERR_TIMEOUT in the same way. */
 prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream);
 
 /* Per-kernel timing hook for benchmarks.  While enabled, every kernel launched

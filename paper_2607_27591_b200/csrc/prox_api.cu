@@ -59,6 +59,10 @@ struct prox_ffn {
   int use_fused;            // batch-1 forward runs as one persistent kernel
   int use_union;            // batch > 1 reads weights once for the union of the tokens' masks
   unsigned long long* trace;  // optional phase time stamps of the persistent kernel (debug)
+  unsigned spin_limit;      // polls after which a device-side wait gives up
+  unsigned bar_bias;        // test knob: keeps the grid barrier of the persistent kernel from completing
+  int* host_flag;           // pinned, mapped word the kernels set when a wait expires
+  int* host_flag_dev;
   // batch > 1: unions of the tokens' masks (allocated when max_batch > 1)
   int* u_in; int* u_ch;     // [D], [F] ascending union lists
   int* u_cnt;               // [0] union inputs, [1] union channels
@@ -503,7 +507,7 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   if (pl.nslots < 3) return pl;
   // the proxy GEMV keeps 16 tensor-memory columns per supergroup (4 scale groups), two sets of up to 256
   if ((D / h->group + 3) / 4 > kMaxSuper) return pl;
-  pl.pstages = (pl.big_bytes - 1024) / kPStageBytes;
+  pl.pstages = (pl.big_bytes - 1024 - 3072) / kPStageBytes;
   if (pl.pstages > kPStages) pl.pstages = kPStages;
   if (pl.pstages < kPStages) return pl;                                   // every loader warp owns a stage
   if (pl.big_bytes < 4 * D * 4) return pl;                                // partial y vectors of the down projection
@@ -577,6 +581,7 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.out_fp32 = h->cfg.out_dtype;
   prm.pstages = pl.pstages;
   prm.scores = h->scores; prm.ghist = h->syncbuf; prm.idx_out = h->idx_x;
+  prm.spin_limit = h->spin_limit; prm.bar_bias = h->bar_bias; prm.host_flag = h->host_flag_dev;
   prm.sel_out = sel_out; prm.yacc = h->yacc;
   prm.bar_count = reinterpret_cast<unsigned long long*>(h->syncbuf + 2048); prm.done_ticket = h->syncbuf + 2050;
   prm.status = h->dev_status;
@@ -621,6 +626,25 @@ prox_status_t forward_kernels(prox_ffn* h, const void* x, int B, int k1, int k2,
   if ((s = launch_channel_select(h, h->scores, B, k2, 0.f, 0, h->sel, F, nullptr, st)) != PROX_OK) return s;
   if (h->use_union && batch_path_ok(h, B)) return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, false);
   return launch_stage2(h, x, B, h->sel, F, nullptr, k2, y, st);
+}
+
+// A block gave up on a wait: counters shared between blocks may be left half-way.  Put every one of
+// them back to its idle state (the stream is idle when this runs).
+prox_status_t reset_shared_state(prox_ffn* h, cudaStream_t st) {
+  const int ns_max = nstrips_for(h->cfg.d_ff, 8);
+  CK(cudaMemsetAsync(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned), st));
+  CK(cudaMemsetAsync(h->ticket, 0, (size_t)h->cfg.max_batch * ns_max * sizeof(unsigned), st));
+  CK(cudaMemsetAsync(h->yacc, 0, (size_t)h->cfg.max_batch * h->cfg.d_model * sizeof(float), st));
+  if (h->gacc) {                               // accumulators of the tensor-core batch path (kept at zero between calls)
+    const size_t F = (size_t)h->cfg.d_ff;
+    CK(cudaMemsetAsync(h->gacc, 0, ((F + 15) / 16) * 256 * sizeof(float), st));
+    CK(cudaMemsetAsync(h->pacc, 0, (F / 64) * 1024 * sizeof(float), st));
+    CK(cudaMemsetAsync(h->cmask, 0, ((F + 3) / 4) * sizeof(unsigned), st));
+    h->cmask_marked = 0;
+  }
+  CK(cudaStreamSynchronize(st));
+  if (h->host_flag) *h->host_flag = 0;
+  return PROX_OK;
 }
 
 }  // namespace
@@ -694,6 +718,11 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   }
   A(cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
   A(cudaDeviceGetAttribute(&h->coop, cudaDevAttrCooperativeLaunch, h->device));
+  h->spin_limit = kSpinLimit;
+  if (st == PROX_OK) {
+    A(cudaHostAlloc(reinterpret_cast<void**>(&h->host_flag), sizeof(int), cudaHostAllocMapped));
+    if (st == PROX_OK) { *h->host_flag = 0; A(cudaHostGetDevicePointer(reinterpret_cast<void**>(&h->host_flag_dev), h->host_flag, 0)); }
+  }
   h->use_fused = 1;
   h->use_union = 1;
   h->use_mma = 1;
@@ -719,6 +748,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
   cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->cmask); cudaFree(h->umask);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
+  if (h->host_flag) cudaFreeHost(h->host_flag);
   if (h->prof) {
     for (auto& r : *h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete h->prof;
@@ -1010,7 +1040,7 @@ prox_status_t prox_ffn_last_mask(prox_ffn_t* h, int B, int k2, int32_t* sel_dev,
   if (B == 1 && h->sel_unordered) {
     // the persistent kernel lists the kept channels in its own order; the score buffer is free between calls
     LaunchScope ls(h, kKChannel, st);
-    mask_ascending_kernel<<<1, 1024, 0, st>>>(h->sel, k2, h->cfg.d_ff, reinterpret_cast<int*>(h->scores), sel_dev);
+    mask_ascending_kernel<<<1, 1024, 0, st>>>(h->sel, k2, h->cfg.d_ff, reinterpret_cast<int*>(h->hbuf), sel_dev);
     CK(cudaGetLastError());
     return PROX_OK;
   }
@@ -1042,6 +1072,12 @@ prox_status_t prox_ffn_forward_host(prox_ffn_t* h, const void* x_host, int B, in
   if (s != PROX_OK) return s;
   if (!y_direct) CK(cudaMemcpyAsync(y_host, h->y_stage, ybytes, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  if (h->host_flag && *reinterpret_cast<volatile int*>(h->host_flag)) {
+    // a bounded device-side wait ran out: y_host is undefined; put the shared counters back and say so
+    CK(cudaMemsetAsync(h->dev_status, 0, sizeof(int), st));
+    s = reset_shared_state(h, st);
+    return s != PROX_OK ? s : PROX_ERR_TIMEOUT;
+  }
   return PROX_OK;
 }
 
@@ -1279,21 +1315,25 @@ prox_status_t prox_last_device_status(prox_ffn_t* h, int32_t* code, void* stream
   CK(cudaMemsetAsync(h->dev_status, 0, sizeof(int), st));
   CK(cudaStreamSynchronize(st));
   if (*code & kWaitExpired) {
-    // A block gave up on a wait: counters shared between blocks may be left
-    // half-way.  Put every one of them back to its idle state.
-    const int ns_max = nstrips_for(h->cfg.d_ff, 8);
-    CK(cudaMemsetAsync(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned), st));
-    CK(cudaMemsetAsync(h->ticket, 0, (size_t)h->cfg.max_batch * ns_max * sizeof(unsigned), st));
-    CK(cudaMemsetAsync(h->yacc, 0, (size_t)h->cfg.max_batch * h->cfg.d_model * sizeof(float), st));
-    if (h->gacc) {                               // accumulators of the tensor-core batch path (kept at zero between calls)
-      const size_t F = (size_t)h->cfg.d_ff;
-      CK(cudaMemsetAsync(h->gacc, 0, ((F + 15) / 16) * 256 * sizeof(float), st));
-      CK(cudaMemsetAsync(h->pacc, 0, (F / 64) * 1024 * sizeof(float), st));
-      CK(cudaMemsetAsync(h->cmask, 0, ((F + 3) / 4) * sizeof(unsigned), st));
-      h->cmask_marked = 0;
-    }
-    CK(cudaStreamSynchronize(st));
+    const prox_status_t s = reset_shared_state(h, st);
+    return s != PROX_OK ? s : PROX_ERR_TIMEOUT;
   }
+  return PROX_OK;
+}
+
+prox_status_t prox_debug_set_wait(prox_ffn_t* h, uint32_t spin_limit, uint32_t barrier_bias) {
+  if (!h) return PROX_ERR_INVALID_ARG;
+  h->spin_limit = spin_limit ? spin_limit : kSpinLimit;
+  h->bar_bias = barrier_bias;
+  return PROX_OK;
+}
+
+prox_status_t prox_ffn_last_stage1(prox_ffn_t* h, int k1, int32_t* idx_dev, float* scores_dev, void* stream) {
+  if (!h || (!idx_dev && !scores_dev)) return PROX_ERR_INVALID_ARG;
+  if (idx_dev && (k1 < 1 || k1 > h->cfg.d_model)) return PROX_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (idx_dev) CK(cudaMemcpyAsync(idx_dev, h->idx_x, (size_t)k1 * sizeof(int), cudaMemcpyDeviceToDevice, st));
+  if (scores_dev) CK(cudaMemcpyAsync(scores_dev, h->scores, (size_t)h->cfg.d_ff * sizeof(float), cudaMemcpyDeviceToDevice, st));
   return PROX_OK;
 }
 

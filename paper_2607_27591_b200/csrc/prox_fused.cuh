@@ -60,6 +60,9 @@ struct FusedParams {
   int pstages;        // stages of the proxy ring that fit (<= kPStages)
   float* scores; unsigned* ghist; int* sel_out;
   int* idx_out;       // the kept input list as this kernel built it (block 0 writes it; for checking)
+  unsigned spin_limit;        // polls after which a device-side wait gives up
+  unsigned bar_bias;          // test knob: added to the grid barrier's target (0 in normal use)
+  int* host_flag;             // mapped host word set to 1 when a wait expires (NULL = none)
   float* yacc; unsigned long long* bar_count; unsigned* done_ticket; int* status;
   int big_bytes;      // bytes of the large shared buffer
   int nslots;         // ring slots of D*2 bytes inside it
@@ -148,11 +151,11 @@ __device__ __forceinline__ void consumer_sync() {     // the 512 consumer thread
 
 // Bounded wait on an mbarrier phase.  Gives up (and raises the block's abort
 // flag) after kSpinLimit polls; once the flag is up every wait returns at once.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned limit = kSpinLimit) {
   if (mbar_try_wait(bar, parity)) return true;
   if (*abort_flag) return false;
 #pragma unroll 1
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
+  for (unsigned it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 256) __nanosleep(64);
     if ((it & 255u) == 255u && *abort_flag) return false;
@@ -166,18 +169,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // warp first waits (bounded) until the consumer of the previous use has seen
 // its data complete; from then on the barrier can only be in phase `use`.
 __device__ __forceinline__ bool slot_wait(uint32_t bar, volatile unsigned* seen, unsigned use,
-                                          volatile int* abort_flag) {
+                                          volatile int* abort_flag, unsigned limit) {
   if (use > 0 && *seen < use) {
     bool ok = false;
 #pragma unroll 1
-    for (unsigned it = 0; it < kSpinLimit; ++it) {
+    for (unsigned it = 0; it < limit; ++it) {
       if (*seen >= use) { ok = true; break; }
       if (it > 256) __nanosleep(32);
       if ((it & 255u) == 255u && *abort_flag) return false;
     }
     if (!ok) { *abort_flag = 1; return false; }
   }
-  if (!mbar_wait(bar, use & 1u, abort_flag)) return false;
+  if (!mbar_wait(bar, use & 1u, abort_flag, limit)) return false;
   *seen = use + 1u;
   return true;
 }
@@ -284,6 +287,9 @@ struct FusedSmem {
   int sstart[kMaxSuper + 2];             // first kept row of every supergroup (and k1)
   int bstart[kMaxSuper + 2];             // first 32-row block of every supergroup (and the block count)
   float soff[4 * kMaxSuper];             // per scale group: code offset (8 or 128) * sum of the kept x, as integers
+  int gstart[4 * kMaxSuper + 2];         // first kept row of every scale group (and k1)
+  unsigned soff_cnt;                     // warps that have finished their share of soff
+  unsigned wmax[32];
   float nsum[kFusedWarps][2];     // RMSNorm: the warps' sums of squares (hi, lo)
   float ninv[2];                  // ... and 1 / sqrt(mean + eps) (hi, lo)
 };
@@ -309,6 +315,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   const int G = gridDim.x, cta = blockIdx.x;
   volatile int* abortp = &sm.abort_flag;
   const unsigned lt_mask = (1u << lane) - 1u;
+  const unsigned spin = p.spin_limit;
 
   // ------------------------------------------------------------------ set-up
   PROX_TRACE(0);
@@ -323,6 +330,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     if (tid == 0) mbar_init(smem_u32(&sm.acc_bar), kFusedConsumerWarps);
     fence_mbar_init();
   }
+  if (tid == 0) sm.soff_cnt = 0;
   if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
   if (tid < kMaxSlots) sm.slot_use[tid] = 0;
   if (NORM) {
@@ -397,6 +405,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   PROX_TRACE(1);
 
   // ------------------------------------------------- A: input mask (top-k1 of |x|)
+  int ebase = 1;
+  const bool per_row_a = p.gshift >= 31;
   {
     const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
     const bool all = THRESH ? (p.tkey_x == 0u) : (k1 >= D);
@@ -436,7 +446,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     // in front (one warp scan plus the totals of the warps in front).
     const int ngrp = D / 8, gpt = (ngrp + kFusedConsumers - 1) / kFusedConsumers;
     const int g0 = min(ngrp, tid * gpt), g1 = (tid < kFusedConsumers) ? min(ngrp, g0 + gpt) : g0;
-    unsigned cnt = 0;
+    unsigned cnt = 0, mk = 0;
 #pragma unroll 1
     for (int g = g0; g < g1; ++g) {
       const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
@@ -445,12 +455,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       for (int e = 0; e < 8; ++e) {
         const unsigned key = (w4[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
         cnt += ((all || key > T) ? 1u : 0u) | ((!all && key == T) ? 0x10000u : 0u);
+        mk = max(mk, key);
       }
     }
     const unsigned inc = warp_scan_incl(cnt, lane);
-    if (lane == 31) sm.wsum[warp] = inc;
+    mk = __reduce_max_sync(0xffffffffu, mk);
+    if (lane == 31) { sm.wsum[warp] = inc; sm.wmax[warp] = mk; }
     __syncthreads();
     PROX_TRACE(14);
+    mk = __reduce_max_sync(0xffffffffu, (lane < kFusedWarps) ? sm.wmax[lane] : 0u);
+    ebase = max(max((int)(mk >> 7), 1) - 22, 1);
     if (THRESH) {
       k1 = (int)__reduce_add_sync(0xffffffffu, (lane < kFusedWarps) ? (sm.wsum[lane] & 0xffffu) : 0u);
       if (cta == 0 && tid == 0) {
@@ -461,10 +475,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     {
       const unsigned ex = __reduce_add_sync(0xffffffffu, (lane < warp) ? sm.wsum[lane] : 0u) + inc - cnt;
       unsigned rg = ex & 0xffffu, re = ex >> 16;
+      // (also, for the proxy GEMV: where every scale group starts in the list)
+      const int gmask = per_row_a ? 0x7fffffff : ((1 << p.gshift) - 1);
 #pragma unroll 1
       for (int g = g0; g < g1; ++g) {
         const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
         const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
+        if (((g * 8) & gmask) == 0) sm.gstart[per_row_a ? 0 : ((g * 8) >> p.gshift)] = (int)(rg + min(re, quota));
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const unsigned key = (w4[e >> 1] >> ((e & 1) * 16)) & 0x7fffu;
@@ -474,6 +491,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         }
       }
     }
+    if (tid == 0) sm.gstart[per_row_a ? 1 : (D >> p.gshift)] = k1;
     __syncthreads();
   }
 
@@ -501,56 +519,19 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     const int nsuper = (ng + 3) >> 2;
     const int sgshift = per_row ? 31 : p.gshift + 2;
     const uint32_t tbase = sm.tmem_base;
-    int* gstart = reinterpret_cast<int*>(sm.hist2);           // [ng + 1] first kept row of every scale group (and k1)
-    // group starts (lower bound in the ascending index list) and the largest exponent
-    if (tid <= ng) {
-      int lo = 0, hi = k1;
-      if (tid == ng) lo = k1;
-      else {
-        const int lim = per_row ? 0 : (tid << p.gshift);
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if ((int)idx16[mid] < lim) lo = mid + 1; else hi = mid; }
-      }
-      gstart[tid] = lo;
+    // supergroup starts and blocks (one warp), the groups' offsets, the block's own score histogram
+    if (warp == 0) {
+      const int r0s = sm.gstart[min(4 * lane, ng)], r1s = sm.gstart[min(4 * lane + 4, ng)];
+      const unsigned nb = lane < nsuper ? (unsigned)((r1s - r0s + 31) >> 5) : 0u;
+      const unsigned incb = warp_scan_incl(nb, lane);
+      if (lane <= nsuper) { sm.sstart[lane] = r0s; sm.bstart[lane] = (int)(incb - nb); }
     }
-    unsigned mk = 0;
-    {
-      const uint32_t* xs32 = reinterpret_cast<const uint32_t*>(xs);
 #pragma unroll 1
-      for (int i = tid; i < D / 2; i += NT) { const uint32_t w = xs32[i]; mk = max(mk, max(w & 0x7fffu, (w >> 16) & 0x7fffu)); }
-    }
-    mk = __reduce_max_sync(0xffffffffu, mk);
-    if (lane == 0) sm.wsum[warp] = mk;
-    __syncthreads();
-    mk = __reduce_max_sync(0xffffffffu, lane < kFusedWarps ? sm.wsum[lane] : 0u);
-    const int emax = max((int)(mk >> 7), 1);
-    const int ebase = max(emax - 22, 1);
-    if (tid == 0) {
-      int acc = 0;
-      for (int s2 = 0; s2 <= nsuper; ++s2) {
-        const int r = gstart[min(4 * s2, ng)];
-        sm.sstart[s2] = r;
-        if (s2 > 0) { sm.bstart[s2 - 1] = acc; acc += (r - sm.sstart[s2 - 1] + 31) >> 5; }
-      }
-      sm.bstart[nsuper] = acc;
-    }
-    // per scale group: offset * sum of the kept x as integers (a warp per group, no atomics)
-#pragma unroll 1
-    for (int g = warp; g < ng; g += kFusedWarps) {
-      int d0 = 0, d1 = 0, d2 = 0, d3 = 0;
-#pragma unroll 1
-      for (int r = gstart[g] + lane; r < gstart[g + 1]; r += 32) {
-        const uint32_t dg = x_digits(xs[idx16[r]], ebase);
-        d0 += (int)(int8_t)(dg & 0xffu); d1 += (int)(int8_t)((dg >> 8) & 0xffu);
-        d2 += (int)(int8_t)((dg >> 16) & 0xffu); d3 += (int)(int8_t)(dg >> 24);
-      }
-      d0 = __reduce_add_sync(0xffffffffu, d0); d1 = __reduce_add_sync(0xffffffffu, d1);
-      d2 = __reduce_add_sync(0xffffffffu, d2); d3 = __reduce_add_sync(0xffffffffu, d3);
-      if (lane == 0) sm.soff[g] = (LO ? 8.f : 128.f) * digits_to_float((uint32_t)d0, (uint32_t)d1, (uint32_t)d2, (uint32_t)d3);
-    }
+    for (int i = tid; i < 512; i += NT) reinterpret_cast<uint4*>(sm.hist)[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     const int nblk = sm.bstart[nsuper];
     const uint32_t ring = (big_u32 + 1023u) & ~1023u;
-    float* red = reinterpret_cast<float*>(sm.hist);           // [3][128][2] partial sums of warps 4..15
+    float* red = reinterpret_cast<float*>(big + (ring - big_u32) + (uint32_t)(kPStages * kPStageBytes));   // [3][128][2] partial sums of warps 4..15
     PROX_TRACE(29);
     if (warp < kFusedConsumerWarps) {
       // a warp owns one stage of the ring: it fills it and issues the stage's MMAs itself (the tensor core
@@ -571,19 +552,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         // ---- scales of this thread's byte column for the groups it will read back
         const int chunk = tile * 8 + (col >> 4);
         const bool col_ok = chunk < nchunks;
-        uint32_t scl[16];
-#pragma unroll
-        for (int it = 0; it < 4; ++it)
-#pragma unroll
-          for (int gq = 0; gq < 4; ++gq) {
-            const int g = 4 * (part + 4 * it) + gq;
-            uint32_t v = 0;
-            if (col_ok && g < ng) {
-              if (LO) v = __ldg(reinterpret_cast<const uint32_t*>(p.S + ((size_t)g * nchunks + chunk) * 32) + (col & 15));
-              else v = (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(p.S + ((size_t)g * nchunks + chunk) * 16) + (col & 15));
-            }
-            scl[it * 4 + gq] = v;
-          }
         const bool c_ok = tile * 8 + c < nchunks;
         bool alive_b = true;
         int sg = 0;
@@ -608,7 +576,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             const int slot = per_row ? 0 : ((i >> p.gshift) & 3);
             brow.x = slot == 0 ? dg : 0u; brow.y = slot == 1 ? dg : 0u; brow.z = slot == 2 ? dg : 0u; brow.w = slot == 3 ? dg : 0u;
           }
-          const bool free_ok = uses == 0 || mbar_wait(my_empty, (uses - 1u) & 1u, abortp);
+          const bool free_ok = uses == 0 || mbar_wait(my_empty, (uses - 1u) & 1u, abortp, spin);
           if (!__all_sync(0xffffffffu, free_ok)) { alive_b = false; break; }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -635,37 +603,56 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         __syncwarp();
         PROX_TRACE(24);
         // ---- read the accumulators back: thread = byte column, warp part p takes supergroups p, p + 4, ...
-        const bool acc_ok = __all_sync(0xffffffffu, alive_b && mbar_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u, abortp));
+        // (the four groups' scales of this byte column: gate / up scales sit in the order of the bytes)
+        auto load_scales = [&](int sgq, uint32_t* dst) {
+#pragma unroll
+          for (int gq = 0; gq < 4; ++gq) {
+            const int g = 4 * sgq + gq;
+            dst[gq] = 0u;
+            if (col_ok && g < ng) {
+              if (LO) dst[gq] = __ldg(reinterpret_cast<const uint32_t*>(p.S + ((size_t)g * nchunks + chunk) * 32) + (col & 15));
+              else dst[gq] = (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(p.S + ((size_t)g * nchunks + chunk) * 16) + (col & 15));
+            }
+          }
+        };
+        uint32_t scn[4];
+        load_scales(part, scn);
+        const bool acc_ok = __all_sync(0xffffffffu, alive_b && mbar_wait(smem_u32(&sm.acc_bar), (unsigned)tile_iter & 1u, abortp, spin));
         tc_fence_after();
+        if (tile_iter == 0) {                  // the groups' offsets come from the four warps that do not load
+#pragma unroll 1
+          for (unsigned it = 0; *reinterpret_cast<volatile unsigned*>(&sm.soff_cnt) < (unsigned)kFusedProducers && it < spin; ++it) __nanosleep(32);
+          __threadfence_block();
+        }
         PROX_TRACE(25);
         float t0 = 0.f, t1 = 0.f;              // 4-bit: sums of the low / high nibble's channel; 8-bit: t0 only
         const bool more = tile + G < ntiles;
+#pragma unroll 1
+        for (int sgd = part; sgd < nsuper; sgd += 4) {
+          if (!acc_ok) break;
+          uint32_t a[16], l[16];
+          const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(16 * sgd);
+          tmem_ld16(ta, a);
+          if (LO) tmem_ld16(ta + 256u, l);
+          uint32_t sc4[4];
 #pragma unroll
-        for (int it = 0; it < 4; ++it) {
-          const int sgd = part + 4 * it;
-          if (sgd < nsuper && acc_ok) {        // warp-uniform
-            uint32_t a[16], l[16];
-            const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(16 * sgd);
-            tmem_ld16(ta, a);
-            if (LO) tmem_ld16(ta + 256u, l);
-            tmem_ld_wait();
-            if (more) { tmem_st16_zero(ta); if (LO) tmem_st16_zero(ta + 256u); }
+          for (int gq = 0; gq < 4; ++gq) sc4[gq] = scn[gq];
+          load_scales(sgd + 4, scn);           // the next round's scales are on their way during this one
+          tmem_ld_wait();
+          if (more) { tmem_st16_zero(ta); if (LO) tmem_st16_zero(ta + 256u); }
 #pragma unroll
-            for (int gq = 0; gq < 4; ++gq) {
-              const int g = 4 * sgd + gq;
-              if (g < ng) {
-                const float off = sm.soff[g];
-                const float fa = digits_to_float(a[4 * gq], a[4 * gq + 1], a[4 * gq + 2], a[4 * gq + 3]);
-                if (LO) {
-                  const float fl = digits_to_float(l[4 * gq], l[4 * gq + 1], l[4 * gq + 2], l[4 * gq + 3]);
-                  const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&scl[it * 4 + gq]));
-                  t0 = fmaf(sc.x, fl - off, t0);
-                  t1 = fmaf(sc.y, fmaf(fa - fl, 0.0625f, -off), t1);
-                } else {
-                  const float sc = __half2float(__ushort_as_half((unsigned short)scl[it * 4 + gq]));
-                  t0 = fmaf(sc, fa - off, t0);
-                }
-              }
+          for (int gq = 0; gq < 4; ++gq) {
+            const int g = 4 * sgd + gq;
+            const float off = sm.soff[min(g, ng - 1)];
+            const float fa = digits_to_float(a[4 * gq], a[4 * gq + 1], a[4 * gq + 2], a[4 * gq + 3]);
+            if (LO) {
+              const float fl = digits_to_float(l[4 * gq], l[4 * gq + 1], l[4 * gq + 2], l[4 * gq + 3]);
+              const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&sc4[gq]));
+              t0 = fmaf(sc.x, fl - off, t0);
+              t1 = fmaf(sc.y, fmaf(fa - fl, 0.0625f, -off), t1);
+            } else {
+              const float sc = __half2float(__ushort_as_half((unsigned short)sc4[gq]));
+              t0 = fmaf(sc, fa - off, t0);
             }
           }
         }
@@ -685,13 +672,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
               const int ch = chunk * 16 + 2 * (col & 7);
               const float s0 = fabsf(u0 * silu_fast(t0)), s1 = fabsf(u1 * silu_fast(t1));
               __stcg(reinterpret_cast<float2*>(p.scores + ch), make_float2(s0, s1));
-              atomicAdd(p.ghist + (__float_as_uint(s0) >> 20), 1u);
-              atomicAdd(p.ghist + (__float_as_uint(s1) >> 20), 1u);
+              atomicAdd(&sm.hist[__float_as_uint(s0) >> 20], 1u);
+              atomicAdd(&sm.hist[__float_as_uint(s1) >> 20], 1u);
             } else {
               const int ch = chunk * 8 + (col & 7);
               const float s0 = fabsf(u0 * silu_fast(t0));
               __stcg(p.scores + ch, s0);
-              atomicAdd(p.ghist + (__float_as_uint(s0) >> 20), 1u);
+              atomicAdd(&sm.hist[__float_as_uint(s0) >> 20], 1u);
             }
           }
         }
@@ -706,9 +693,40 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         }
       }
     }
+    else {
+      // Blocks without a tile pull the kept rows into L2 (whole rows, one bulk prefetch each): the loader
+      // warps of the other blocks then find them there instead of waiting for HBM one by one.
+      if (cta >= ntiles && lane < 8) {
+        const int nidle = G - ntiles, slot_i = (cta - ntiles) * (kFusedProducers * 8) + (warp - kFusedConsumerWarps) * 8 + lane;
+#pragma unroll 1
+        for (int r = slot_i; r < k1; r += nidle * kFusedProducers * 8)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.P + (size_t)idx16[r] * (size_t)row_bytes), "r"((uint32_t)row_bytes) : "memory");
+      }
+      // the other four warps: per scale group, offset * sum of the kept x as integers (for the codes' offset binary)
+#pragma unroll 1
+      for (int g = warp - kFusedConsumerWarps; g < ng; g += kFusedProducers) {
+        int d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+#pragma unroll 1
+        for (int r = sm.gstart[g] + lane; r < sm.gstart[g + 1]; r += 32) {
+          const uint32_t dg = x_digits(xs[idx16[r]], ebase);
+          d0 += (int)(int8_t)(dg & 0xffu); d1 += (int)(int8_t)((dg >> 8) & 0xffu);
+          d2 += (int)(int8_t)((dg >> 16) & 0xffu); d3 += (int)(int8_t)(dg >> 24);
+        }
+        d0 = __reduce_add_sync(0xffffffffu, d0); d1 = __reduce_add_sync(0xffffffffu, d1);
+        d2 = __reduce_add_sync(0xffffffffu, d2); d3 = __reduce_add_sync(0xffffffffu, d3);
+        if (lane == 0) sm.soff[g] = (LO ? 8.f : 128.f) * digits_to_float((uint32_t)d0, (uint32_t)d1, (uint32_t)d2, (uint32_t)d3);
+      }
+      __syncwarp();
+      if (lane == 0) { __threadfence_block(); atomicAdd(&sm.soff_cnt, 1u); }
+    }
     // the tensor memory is not used after this phase
     tc_fence_before();
     __syncthreads();
+    if (cta < ntiles) {
+      // one atomic per occupied bin and block (thousands of single increments on a few hot bins serialise in L2)
+#pragma unroll 1
+      for (int i = tid; i < 2048; i += NT) { const unsigned v = sm.hist[i]; if (v) atomicAdd(p.ghist + i, v); }
+    }
     if (warp == 0) tmem_free_all(tbase);
   }
 
@@ -722,16 +740,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     __threadfence();                          // cumulative: publishes the block's writes seen through the barrier above
     const unsigned long long old = atomicAdd(p.bar_count, 1ull);
     // the count is reset by the host long before 2^32 calls; the low word is enough for the division
-    const unsigned long long target = old - (unsigned long long)((unsigned)old % (unsigned)G) + (unsigned long long)G;
+    const unsigned long long target = old - (unsigned long long)((unsigned)old % (unsigned)G) + (unsigned long long)G +
+                                      (unsigned long long)p.bar_bias;
     bool ok = (old + 1ull == target);
 #pragma unroll 1
-    for (unsigned it = 0; !ok && it < kSpinLimit; ++it) {
+    for (unsigned it = 0; !ok && it < spin; ++it) {
       unsigned long long cur;
       asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(cur) : "l"(p.bar_count) : "memory");
       ok = cur >= target;
       if (!ok && it > 64) __nanosleep(32);
     }
-    if (!ok) { sm.abort_flag = 1; atomicOr(p.status, kWaitExpired); }
+    if (!ok) { sm.abort_flag = 1; atomicOr(p.status, kWaitExpired); if (p.host_flag) *reinterpret_cast<volatile int*>(p.host_flag) = 1; }
     __threadfence();
   }
   __syncthreads();
@@ -1134,7 +1153,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       // wait (bounded) until the consumer warps have listed the block's definite share
       bool go = false;
 #pragma unroll 1
-      for (unsigned it = 0; it < kSpinLimit; ++it) {
+      for (unsigned it = 0; it < spin; ++it) {
         if (*reinterpret_cast<volatile int*>(&sm.go)) { go = true; break; }
         if (*abortp) break;
         __nanosleep(32);
@@ -1166,7 +1185,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
             };
             if (blocked()) {
 #pragma unroll 1
-              for (unsigned it = 0; it < kSpinLimit; ++it) {
+              for (unsigned it = 0; it < spin; ++it) {
                 ready = *reinterpret_cast<volatile int*>(&sm.nready);
                 kdone = *reinterpret_cast<volatile int*>(&sm.keys_done) != 0;
                 cdone = *reinterpret_cast<volatile int*>(&sm.c_done) != 0;
@@ -1175,7 +1194,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
               }
               if (blocked()) { sm.abort_flag = 1; dead = true; break; }
             }
-            if (use > 0 && !mbar_wait(smem_u32(&sm.mbar_empty[slot]), (use - 1u) & 1u, abortp)) { dead = true; break; }
+            if (use > 0 && !mbar_wait(smem_u32(&sm.mbar_empty[slot]), (use - 1u) & 1u, abortp, spin)) { dead = true; break; }
             const uint16_t* src;
             if (q < 2 * nb) {
               src = ((q & 1) ? p.wu : p.wg) + (size_t)sm.mysel[mi] * D;
@@ -1209,8 +1228,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         const unsigned sq = base_seq + 2u * (unsigned)c;
         const int sg = (int)(sq % (unsigned)NS), su = (int)((sq + 1u) % (unsigned)NS);
         const unsigned ug = sq / (unsigned)NS, uu = (sq + 1u) / (unsigned)NS;
-        const bool ok1 = slot_wait(smem_u32(&sm.mbar_full[sg]), &sm.slot_use[sg], ug, abortp);
-        const bool ok2 = slot_wait(smem_u32(&sm.mbar_full[su]), &sm.slot_use[su], uu, abortp);
+        const bool ok1 = slot_wait(smem_u32(&sm.mbar_full[sg]), &sm.slot_use[sg], ug, abortp, spin);
+        const bool ok2 = slot_wait(smem_u32(&sm.mbar_full[su]), &sm.slot_use[su], uu, abortp, spin);
         float ag = 0.f, au = 0.f, ag2 = 0.f, au2 = 0.f;
         if (ok1 && ok2) {
           const uint32_t pg = big_u32 + (uint32_t)sg * row_bytes2, pu = big_u32 + (uint32_t)su * row_bytes2;
@@ -1249,7 +1268,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           const unsigned sq = base_seq + 2u * (unsigned)nb + (unsigned)c;
           const int sd = (int)(sq % (unsigned)NS);
           const unsigned ud = sq / (unsigned)NS;
-          const bool ok = slot_wait(smem_u32(&sm.mbar_full[sd]), &sm.slot_use[sd], ud, abortp);
+          const bool ok = slot_wait(smem_u32(&sm.mbar_full[sd]), &sm.slot_use[sd], ud, abortp, spin);
           if (ok) {
             const float hv = sm.hval[c];
             const uint32_t pd = big_u32 + (uint32_t)sd * row_bytes2;
@@ -1307,6 +1326,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     // waited for here (bounded) so that none lands after the block has left.
     if (tid == 0) {
       atomicOr(p.status, kWaitExpired);
+      if (p.host_flag) *reinterpret_cast<volatile int*>(p.host_flag) = 1;
       const unsigned issued = sm.prod_seq;
       const unsigned first = issued > (unsigned)NS ? issued - (unsigned)NS : 0u;
       for (unsigned q = first; q < issued; ++q) {        // the latest use of every slot
