@@ -74,6 +74,8 @@ _SIGS = {
     "prox_fused_trace": [_vp, _i, _vp, _i],
     "prox_fused_kernel_info": [_vp, _i, _i, C.POINTER(C.c_int32)],
     "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
+    "prox_ffn_last_stage1": [_vp, _i, _vp, _vp, _vp],
+    "prox_debug_set_wait": [_vp, C.c_uint32, C.c_uint32],
     "prox_profile_enable": [_vp, _i],
     "prox_profile_read": [_vp, C.POINTER(C.c_int64), C.POINTER(_d)],
 }
@@ -285,10 +287,27 @@ def prox_algorithmic_bytes(handle: int, rows_in: int, rows_ch: int):
     return a.value, b.value, c.value, d.value
 
 
-def prox_last_device_status(handle: int, stream=None) -> int:
+def prox_last_device_status_raw(handle: int, stream=None):
+    """(status, code) of prox_last_device_status: status is PROX_ERR_TIMEOUT (6) when bit 4 of code is set."""
     code = C.c_int32()
-    _check(_lib.prox_last_device_status(handle, C.byref(code), _ptr(stream)), "prox_last_device_status")
-    return code.value
+    status = _lib.prox_last_device_status(handle, C.byref(code), _ptr(stream))
+    return status, code.value
+
+
+def prox_last_device_status(handle: int, stream=None) -> int:
+    """The status word (bit 4 = a bounded wait expired; the library has then reset its shared counters)."""
+    status, code = prox_last_device_status_raw(handle, stream)
+    if status not in (0, 6):
+        _check(status, "prox_last_device_status")
+    return code
+
+
+def prox_ffn_last_stage1(handle: int, k1: int, idx=None, scores=None, stream=None) -> None:
+    _check(_lib.prox_ffn_last_stage1(handle, k1, _ptr(idx), _ptr(scores), _ptr(stream)), "prox_ffn_last_stage1")
+
+
+def prox_debug_set_wait(handle: int, spin_limit: int, barrier_bias: int) -> None:
+    _check(_lib.prox_debug_set_wait(handle, spin_limit, barrier_bias), "prox_debug_set_wait")
 
 
 def prox_launch_count(handle: int) -> int:

@@ -591,7 +591,8 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   if (taus) {
     // |x| >= tau_x  <=>  15-bit bf16 magnitude >= ceil(bits(tau_x) / 2^16);  score >= tau_s  <=>  bits >= bits
     uint32_t bx, bs;
-    std::memcpy(&bx, &taus[0], 4); std::memcpy(&bs, &taus[1], 4);
+    const float tx = std::fabs(taus[0]), ts = std::fabs(taus[1]);        // -0.0f is the threshold 0
+    std::memcpy(&bx, &tx, 4); std::memcpy(&bs, &ts, 4);
     prm.tkey_x = (bx >> 16) + ((bx & 0xffffu) ? 1u : 0u);
     prm.tkey_s = bs;
     prm.cnt_x_out = h->cnt_x; prm.count_out = h->cnt_s; prm.counters = h->counters;
@@ -1277,7 +1278,7 @@ prox_status_t prox_pack_load(prox_ffn_t* h, const char* path, void* stream) {
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   const bool shape_ok = hd.d_model == D && hd.d_ff == F && (hd.bits == 4 || hd.bits == 8 || hd.bits == 16) &&
                         (hd.group == D || hd.group == 128);
-  if (!shape_ok) { std::fclose(f); return PROX_ERR_INVALID_ARG; }
+  if (!shape_ok || (hd.bits == 16 && hd.group != D)) { std::fclose(f); return PROX_ERR_INVALID_ARG; }   // 16-bit proxies have no groups
   prox_status_t s = alloc_packed(h, hd.bits, hd.group);
   if (s != PROX_OK) { std::fclose(f); free_packed(h); return s; }
   const int ngroups = D / hd.group;

@@ -1,6 +1,5 @@
 """GPU parity: libprox (through the C ABI) against the CPU oracle, element by
-element on the same seeded inputs.  Tolerances (written here, derived in
-the design doc): integer work (quantizer codes, input mask) bit-exact; channel masks
+element on the same seeded inputs.  Tolerances (written here): integer work (quantizer codes, input mask) bit-exact; channel masks
 identical outside a 1e-3 relative band around the k2-th oracle score; outputs
 within 2e-2 * RMS(y_oracle)."""
 import numpy as np
@@ -197,6 +196,74 @@ def _forward_check(pb, p, t, k1, k2, B=1):
         y_ref, _ = po.stage2(p.x[t + b], used_np[b], p.wg, p.wu, p.wd)
         check_y(y_np[b], y_ref)
     return nd
+
+
+def _check_fused_stage1(pb, p, tx, x64, k1, k2):
+    """The persistent kernel's own kept-input list and proxy scores against the oracle."""
+    y = p.y_empty()
+    pb.prox_ffn_forward(p.h, tx, 1, k1, k2, y)
+    idx = torch.empty(k1, dtype=torch.int32, device="cuda")
+    sc = torch.empty(p.F, dtype=torch.float32, device="cuda")
+    pb.prox_ffn_last_stage1(p.h, k1, idx, sc)
+    torch.cuda.synchronize()
+    dg, du, _ = p.deq[p.fmt]
+    idx_ref = po.input_topk(x64, k1)
+    assert np.array_equal(idx.cpu().numpy().astype(np.int64), idx_ref), "kept inputs differ from the oracle"
+    score = po.proxy_scores(x64, idx_ref, dg, du)
+    _, thr = po.channel_topk(score, k2)
+    err = float(np.max(np.abs(sc.cpu().numpy().astype(np.float64) - score)) / thr)
+    assert err < 2e-4, err                # relative to the threshold score (fp32 sums, fast exp)
+    return err
+
+
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0), (8, 128)])
+def test_fused_kernel_own_input_list_and_scores(pb, toy, bits, group):
+    wl, p = toy
+    p.quantize(bits, group)
+    k1, k2 = wl.points[50]
+    for t in (0, 7, 19):
+        _check_fused_stage1(pb, p, p.t_x[t], p.x[t], k1, k2)
+    # hand-made ties among the magnitudes: the lower index must win inside the kernel too
+    from tests.gpu_common import dev_bf16
+    vals = np.array([1.0, -1.0, 0.5, 2.0, -2.0, 0.0, -0.0, 1.0], dtype=np.float32)
+    x = np.tile(vals, p.D // 8)[None, :]
+    tx = dev_bf16(inputs.f32_to_bf16_bits(x))
+    for k1t in (1, 64, 65, 129, 300, p.D - 3):
+        _check_fused_stage1(pb, p, tx, x[0].astype(np.float64), k1t, k2)
+    # inputs spread over many binades (the integer form of x drops bits only far below the largest)
+    xf = p.x[3].copy()
+    xf[::7] *= 2.0 ** -20
+    xf[5::11] *= 2.0 ** 9
+    bits16 = inputs.f32_to_bf16_bits(xf.astype(np.float32)[None, :])
+    _check_fused_stage1(pb, p, dev_bf16(bits16), po.bf16_to_f64(bits16)[0], k1, k2)
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+def test_bounded_wait_runs_out_and_the_handle_recovers(pb, toy):
+    """A grid barrier that cannot complete: every block gives up after a few hundred polls and leaves
+    (nothing hangs, nothing faults); y is not written, the status says so, and the next call is ordinary."""
+    wl, p = toy
+    p.quantize(4, 128)
+    k1, k2 = wl.points[50]
+    y = torch.full((1, p.D), 7.0, dtype=torch.float32, device="cuda")
+    pb.prox_debug_set_wait(p.h, 300, 1)
+    try:
+        pb.prox_ffn_forward(p.h, p.t_x[1], 1, k1, k2, y)
+        torch.cuda.synchronize()
+        status, code = pb.prox_last_device_status_raw(p.h)
+        assert code & 4 and status == 6          # PROX_ERR_TIMEOUT
+        assert torch.all(y == 7.0)               # untouched
+        # the host-buffer entry point synchronises and reports the expiry itself
+        xh = torch.from_numpy(p.bits["x"][1:2].view(np.int16)).view(torch.bfloat16).pin_memory()
+        yh = torch.empty(1, p.D, dtype=torch.float32).pin_memory()
+        with pytest.raises(pb.ProxError) as ei:
+            pb.prox_ffn_forward_host(p.h, xh, 1, k1, k2, yh)
+        assert ei.value.status == 6
+    finally:
+        pb.prox_debug_set_wait(p.h, 0, 0)
+    assert pb.prox_last_device_status(p.h) == 0
+    _forward_check(pb, p, 1, k1, k2)
+    assert pb.prox_last_device_status(p.h) == 0
 
 
 def test_forward_toy_all_tokens(pb, toy):
@@ -714,6 +781,8 @@ def test_forms_on_odd_shapes(pb, D, F, bits, group):
             k1 = int(rng.integers(1, D + 1))
             k2 = int(rng.integers(1, F + 1))
             t = trial % 4
+            # the persistent kernel's own input list and scores at this shape and budget
+            _check_fused_stage1(pb, p, p.t_x[t], p.x[t], k1, k2)
             # layer sub-block, top-k
             x_res = (p.x[t] * 1.3).astype(np.float32)[None, :]
             t_x = torch.from_numpy(x_res).cuda()

@@ -64,6 +64,21 @@ def test_qwen3_8b(pb):
     _run(pb, "qwen3_8b", 4, [((4, 128), 70)])
 
 
+@pytest.mark.parametrize("name,fmt", [("qwen3_8b", (4, 128)), ("llama3_8b", (8, 0)), ("llama3_70b", (4, 0))])
+def test_fused_kernel_own_input_list_and_scores_at_bench_shapes(pb, name, fmt):
+    from tests.test_gpu_parity import _check_fused_stage1
+    wl, wg, wu, wd, x = inputs.make_workload(name, n_tokens=2)
+    p = Problem(pb, wg, wu, wd, x)
+    try:
+        p.quantize(*fmt)
+        k1, k2 = wl.points[70]
+        for t in range(2):
+            _check_fused_stage1(pb, p, p.t_x[t], p.x[t], k1, k2)
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
+
+
 def test_llama3_8b_formats_and_batches(pb):
     _run(pb, "llama3_8b", 8, [((8, 0), 70), ((4, 128), 70), ((4, 128), 40)], batches=(1, 4, 8))
 
@@ -77,7 +92,7 @@ def test_llama3_70b_s1_sweep(pb):
     p = Problem(pb, wg, wu, wd, x)
     try:
         p.quantize(4, 0)
-        for k1, k2 in wl.extra["s1_sweep"][::3]:
+        for k1, k2 in wl.extra["s1_sweep"]:
             y = p.y_empty()
             sel = torch.empty(1, k2, dtype=torch.int32, device="cuda")
             pb.prox_ffn_forward(p.h, p.t_x[0], 1, k1, k2, y)
