@@ -51,6 +51,9 @@ def parse():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--small-case", nargs="*", default=None, metavar="ARG",
+                    help="profiler target instead of the benchmark: [workload] [calls] [batch] [topk|threshold|block]; two weight "
+                         "replicas, a handful of launches, < 2 GB on the device")
     ap.add_argument("--alpha", action="store_true",
                     help="also measure the proxy-cost ratio alpha (integer proxy GEMV / 16-bit GEMV at equal input sparsity)")
     return ap.parse_args()
@@ -633,8 +636,61 @@ def run_prox(args):
         dist.destroy_process_group()
 
 
+def run_small_case(argv):
+    """A few calls on one small synthetic problem (two weight replicas): what the ncu captures under profiles/ ran."""
+    import torch
+    from paper_2607_27591_b200 import binding as pb, inputs
+    name = argv[0] if len(argv) > 0 else "qwen3_8b"
+    ncalls = int(argv[1]) if len(argv) > 1 else 6
+    batch = int(argv[2]) if len(argv) > 2 else 1
+    form = argv[3] if len(argv) > 3 else "topk"
+    wl = inputs.WORKLOADS[name]
+    D, F = wl.d_model, wl.d_ff
+    k1, k2 = wl.points[70] if 70 in wl.points else next(iter(wl.points.values()))
+    bits, group = wl.proxies[0]
+    torch.manual_seed(0)
+    replicas, handles = [], []
+    for _ in range(2):
+        w = [(torch.randn(s, device="cuda") * wl.w_std).to(torch.bfloat16) for s in ((F, D), (F, D), (D, F))]
+        replicas.append(w)
+        h = pb.prox_ffn_create(D, F, max(1, batch), 0, *w)
+        pb.prox_quantize_proxy(h, bits, group)
+        handles.append(h)
+    x = torch.randn(8, batch, D, device="cuda").to(torch.bfloat16)
+    y = torch.zeros(8, batch, D, dtype=torch.bfloat16, device="cuda")
+    if form == "threshold":
+        tau_x = float(x[0, 0].float().abs().topk(k1).values[-1])
+        sel = torch.empty(1, F, dtype=torch.int32, device="cuda")
+        cnt = torch.empty(1, dtype=torch.int32, device="cuda")
+        sc = torch.empty(1, F, dtype=torch.float32, device="cuda")
+        taus = []
+        for h in handles:
+            pb.prox_stage1_mask_threshold(h, x[0], 1, tau_x, 0.0, sel, cnt, sc)
+            taus.append(float(sc[0].topk(k2).values[-1]))
+        for t in range(ncalls):
+            pb.prox_ffn_forward_threshold(handles[t % 2], x[t % 8], 1, tau_x, taus[t % 2], y[t % 8])
+    elif form == "block":
+        nw = torch.ones(D, dtype=torch.bfloat16, device="cuda")
+        xr = x[:, 0, :].float().contiguous()
+        for t in range(ncalls):
+            pb.prox_ffn_block_forward(handles[t % 2], xr[t % 8:t % 8 + 1], nw, 1e-6, 1, k1, k2, xr[t % 8:t % 8 + 1])
+        y = xr
+    else:
+        for t in range(ncalls):
+            pb.prox_ffn_forward(handles[t % 2], x[t % 8], batch, k1, k2, y[t % 8])
+    torch.cuda.synchronize()
+    status = [pb.prox_last_device_status(h) for h in handles]
+    print(f"{name}: {ncalls} calls ({form}), batch {batch}, k1={k1} k2={k2}, device status {status}, "
+          f"|y| sum {float(y.float().abs().sum()):.4f}")
+    for h in handles:
+        pb.prox_ffn_destroy(h)
+    sys.exit(0 if not any(status) else 1)
+
+
 def main():
     args = parse()
+    if args.small_case is not None:
+        run_small_case(args.small_case)
     if args.impl == "reference":
         run_reference(args)
     else:

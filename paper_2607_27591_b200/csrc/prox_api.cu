@@ -542,12 +542,25 @@ cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStr
   cfg.blockDim = dim3(kFusedThreads);
   cfg.dynamicSmemBytes = pl.smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  // Cooperative (all blocks co-resident: the kernel has a grid barrier) and, if the driver takes the two
+  // together, programmatic stream serialization: the next launch on the stream is set up while this one
+  // drains, and its blocks wait (griddepcontrol.wait) for this grid to complete before they read anything.
+  static int use_pdl = getenv("PROX_NO_PDL") ? 0 : 1;
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeCooperative;
   at[0].val.cooperative = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, prm);
+  cfg.numAttrs = use_pdl ? 2 : 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, prm);
+  if (e != cudaSuccess && use_pdl) {
+    (void)cudaGetLastError();
+    use_pdl = 0;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, prm);
+  }
+  return e;
 }
 
 template <int BITS, int NG>

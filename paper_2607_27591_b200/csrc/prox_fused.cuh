@@ -333,6 +333,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   if (tid == 0) sm.soff_cnt = 0;
   if (tid == 0) { sm.abort_flag = 0; sm.ncand = 0; sm.ncand2 = 0; sm.prod_seq = 0; sm.next_c = 0; sm.go = 0; }
   if (tid < kMaxSlots) sm.slot_use[tid] = 0;
+  // the launch may have been set up while the previous kernel of the stream was still draining: nothing of
+  // global memory is touched before that kernel has completed
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (NORM) {
     // FFN input = bf16(RMSNorm(residual stream) * norm weight), the correctly rounded value (the masks
     // depend on it).  Every block does all of it; x and w pass through shared memory once.
@@ -426,6 +430,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       unsigned above1;
       const unsigned bin1 = kth_in_block<2, false>(sm.hist, (unsigned)k1, sm.wsum, lane, warp, &above1);
       PROX_TRACE(11);
+      // Inputs whose magnitude lies in a bin above the threshold bin are kept whatever the exact threshold:
+      // their packed proxy rows are pulled into L2 now (every block a share of them, one bulk prefetch per
+      // row), a few microseconds before the proxy GEMV asks for them.
+      if (warp >= kFusedConsumerWarps) {
+        const size_t prow = (size_t)(F / CH) * 16;
+#pragma unroll 1
+        for (int i = cta + (tid - kFusedConsumers) * G; i < D; i += G * 32 * kFusedProducers)
+          if ((((unsigned)xs[i] & 0x7fffu) >> 5) > bin1)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.P + (size_t)i * prow), "r"((uint32_t)prow) : "memory");
+      }
 #pragma unroll 1
       for (int i = tid; i < D / 2; i += NT) {
         const uint32_t w = xs32[i];
