@@ -12,6 +12,7 @@
 #include "prox_kernels.cuh"
 #include "prox_fused.cuh"
 #include "prox_batch_mma.cuh"
+#include "prox_batch_umma.cuh"
 
 using namespace prox;
 
@@ -71,13 +72,17 @@ struct prox_ffn {
   float* hb;                // [F][8]  h of every token at a union channel
   float* gacc;              // [F rounded up to 16][2][8] gate / up pre-activations (tensor-core batch path), kept at zero
   int use_mma;              // batch > 1: Stage 2 and the 4-bit proxy GEMM run on the tensor cores
-  float* pacc;              // [F / 64][128 code columns][8] proxy sums of the tensor-core batch path, kept at zero
+  float* pacc;              // [8 tokens][gate | up][F] proxy sums of the tensor-core batch path, kept at zero
   int mask_policy;          // batch > 1: 0 = every token its own channel mask, 1 = one mask from the summed scores
   int cmask_marked;         // Stage 1 of the running forward call has set the tokens' bits in cmask already
   unsigned* cmask;          // [F / 4] one byte per channel: which tokens kept it (kept at zero between calls)
   uint8_t* umask;           // [F] that byte for every union row
   __half* xh;               // [8][D] masked, scaled fp16 x of the tensor-core proxy GEMM
   float* tokfac;            // [8] per token: what undoes its scaling
+  uint32_t* xd;             // [D][8] digit words of the tokens' masked inputs (tcgen05 proxy GEMM)
+  float* soffb;             // [D / 128][8] per 128-input unit and token: sum of the integer inputs
+  CUtensorMap pmap;         // the packed proxy as a 2-D byte tensor (TMA descriptor of the batched Stage 1)
+  const void* pmap_P; int pmap_row_bytes, pmap_D;   // what pmap was encoded for
   void* x_stage;            // device staging for the host-buffer entry point
   void* y_stage;
   int64_t launches;
@@ -311,22 +316,51 @@ bool stage2_mma_ok(const prox_ffn* h) {
   return h->use_mma && h->gacc && stage2_mma_smem(h) <= (size_t)h->smem_optin - 4096;
 }
 
+// TMA descriptor of the packed proxy rows: bytes [D][row_bytes], box = 128 bytes x 128 rows, 128-byte swizzle
+// (what the integer MMA's A operand wants).  The driver entry point is looked up at run time: the library
+// does not link against the driver.
+prox_status_t ensure_pmap(prox_ffn* h, int row_bytes) {
+  const int D = h->cfg.d_model;
+  if (h->pmap_P == h->P && h->pmap_row_bytes == row_bytes && h->pmap_D == D) return PROX_OK;
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_fn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    CK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr));
+    if (!fn || qr != cudaDriverEntryPointSuccess) return PROX_ERR_UNSUPPORTED;
+    encode = reinterpret_cast<encode_fn>(fn);
+  }
+  const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)D};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  const cuuint32_t box[2] = {128u, 128u}, estr[2] = {1u, 1u};
+  const CUresult r = encode(&h->pmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(h->P), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return PROX_ERR_CUDA;
+  h->pmap_P = h->P; h->pmap_row_bytes = row_bytes; h->pmap_D = D;
+  return PROX_OK;
+}
+
 // mark_mask: also set the tokens' bits in the per-channel bytes that the tensor-core Stage 2 of the
 // SAME call turns into the union (only prox_ffn_forward asks for it: the bytes must be consumed)
 prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int k2, int* sel, int sel_stride,
-                                  float* scores, cudaStream_t st, bool mark_mask = false) {
+                                  float* scores, cudaStream_t st, bool mark_mask = false, bool want_scores = true) {
   h->cmask_marked = 0;
   const int D = h->cfg.d_model, F = h->cfg.d_ff;
   prox_status_t s;
   const int gshift_m = (h->group == D) ? 31 : 7;
-  if (h->use_mma && h->pacc && h->bits == 4 && F % 64 == 0) {
+  if (h->use_mma && h->pacc && (h->bits == 4 || h->bits == 8) && F % 64 == 0) {
     // tensor-core path over all inputs (no union list): per-token masked, scaled fp16 x, then equal
     // ranges of (strip, K-block) units per block, then the per-token channel masks
     const size_t lim = (size_t)h->smem_optin - 16384;
     const bool fast_masks = (size_t)D * 2 <= lim && (size_t)F * 4 <= lim;
     static bool attr_p = false;
     if (!attr_p) {
-      CK(cudaFuncSetAttribute(proxy_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaWarps * 1024 * (int)sizeof(float)));
+      CK(cudaFuncSetAttribute(proxy_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
+      CK(cudaFuncSetAttribute(proxy_umma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
       CK(cudaFuncSetAttribute(batch_input_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
       CK(cudaFuncSetAttribute(batch_channel_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
       attr_p = true;
@@ -334,17 +368,48 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     if (fast_masks) {
       LaunchScope ls(h, kKInput, st);
       batch_input_mask_kernel<<<kBT, kFusedThreads, (size_t)D * 2, st>>>(static_cast<const uint16_t*>(x), B, D, k1,
-                                                                        h->xh, h->tokfac);
+                                                                        h->xh, h->tokfac, h->xd, h->soffb);
     } else {
       if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
       LaunchScope ls(h, kKInput, st);
       proxy_xprep_kernel<<<kBT, 512, 0, st>>>(static_cast<const uint16_t*>(x), h->idx_x, D, k1, B, D, h->xh, h->tokfac);
+      batch_digits_kernel<<<kBT, 512, 0, st>>>(h->xh, D, h->xd, h->soffb);
     }
+    bool direct = false;
     {
       LaunchScope ls(h, kKProxy, st);
-      proxy_mma_kernel<<<h->sm_count, kMmaThreads, (size_t)kMmaWarps * 1024 * sizeof(float), st>>>(
-          h->P, h->S, h->xh, h->tokfac, D, F, gshift_m, h->pacc);
-      proxy_mma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
+      const int row_bytes = (F / ch_per_chunk(h->bits)) * 16, ntiles = (row_bytes + 127) / 128, nunits = D / 128;
+      int usplit = (2 * h->sm_count + ntiles - 1) / ntiles;
+      if (usplit > nunits) usplit = nunits;
+      if (usplit < 1) usplit = 1;
+      const int nitems = ntiles * usplit;
+      const int grid = nitems < h->sm_count ? nitems : h->sm_count;
+      const size_t smem = (size_t)kBuSmem;
+      if ((s = ensure_pmap(h, row_bytes)) != PROX_OK) return s;
+      {
+        // programmatic dependent launch: the kernel sets up and requests its first weight tiles while the
+        // kernel that masks the inputs still runs; it waits for that kernel before it reads anything of this call
+        static int use_pdl = getenv("PROX_NO_PDL") ? 0 : 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kBuThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = use_pdl ? 1 : 0;
+        const __half* Sp = h->S; const uint32_t* xdp = h->xd; const float* sop = h->soffb; const float* tfp = h->tokfac;
+        int Dv = D, Fv = F, gs = gshift_m, us = usplit; float* pa = h->pacc; int* stp = h->dev_status;
+        void* args[] = {&h->pmap, &Sp, &xdp, &sop, &tfp, &Dv, &Fv, &gs, &us, &pa, &stp};
+        const void* fn = h->bits == 4 ? reinterpret_cast<const void*>(&proxy_umma_kernel<4>) : reinterpret_cast<const void*>(&proxy_umma_kernel<8>);
+        cudaError_t e = cudaLaunchKernelExC(&cfg, fn, args);
+        if (e != cudaSuccess && use_pdl) {              // attribute not accepted here: plain launch from now on
+          (void)cudaGetLastError();
+          use_pdl = 0; cfg.numAttrs = 0;
+          e = cudaLaunchKernelExC(&cfg, fn, args);
+        }
+        CK(e);
+      }
+      direct = fast_masks && !want_scores && h->mask_policy == 0;
+      if (!direct) proxy_umma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
     }
     CK(cudaGetLastError());
     if (h->mask_policy == 1) {
@@ -352,7 +417,7 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
       LaunchScope ls(h, kKChannel, st);
       shared_score_kernel<<<(F + 255) / 256, 256, 0, st>>>(scores, B, F, h->svals);
       batch_channel_mask_kernel<<<1, kFusedThreads, (size_t)F * 4, st>>>(h->svals, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr, (1u << B) - 1u);
+                                                                        mark_mask ? h->cmask : nullptr, (1u << B) - 1u, nullptr);
       replicate_mask_kernel<<<(k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B);
       CK(cudaGetLastError());
       if (mark_mask) h->cmask_marked = 1;
@@ -362,7 +427,7 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     {
       LaunchScope ls(h, kKChannel, st);
       batch_channel_mask_kernel<<<B, kFusedThreads, (size_t)F * 4, st>>>(scores, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr, 0u);
+                                                                        mark_mask ? h->cmask : nullptr, 0u, direct ? h->pacc : nullptr);
     }
     CK(cudaGetLastError());
     if (mark_mask) h->cmask_marked = 1;
@@ -632,7 +697,7 @@ prox_status_t forward_kernels(prox_ffn* h, const void* x, int B, int k1, int k2,
   h->sel_unordered = 0;
   if (B > 1 && h->mask_policy == 1 && !(h->use_union && batch_path_ok(h, B, true))) return PROX_ERR_UNSUPPORTED;
   if (h->use_union && batch_path_ok(h, B, true)) {
-    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h))) != PROX_OK) return s;
+    if ((s = launch_stage1_batch(h, x, B, k1, k2, h->sel, F, h->scores, st, stage2_mma_ok(h), false)) != PROX_OK) return s;
     return launch_stage2_batch(h, x, B, h->sel, F, k2, y, st, true);
   }
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
@@ -727,6 +792,7 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
       A(dev_alloc(&h->cmask, (size_t)(F + 3) / 4)); A(dev_alloc(&h->umask, (size_t)F));
       if (st == PROX_OK) A(cudaMemset(h->cmask, 0, (size_t)((F + 3) / 4) * sizeof(unsigned)));
       A(dev_alloc(&h->tokfac, (size_t)kBT));
+      A(dev_alloc(&h->xd, (size_t)D * kBT)); A(dev_alloc(&h->soffb, (size_t)(D / 128) * kBT));
     }
     if (st == PROX_OK) A(cudaMemset(h->gacc, 0, (size_t)((F + 15) / 16) * 256 * sizeof(float)));
   }
@@ -760,7 +826,7 @@ void prox_ffn_destroy(prox_ffn_t* h) {
   cudaFree(h->idx_x); cudaFree(h->cnt_x); cudaFree(h->part); cudaFree(h->ticket);
   cudaFree(h->scores); cudaFree(h->svals); cudaFree(h->xn); cudaFree(h->sel); cudaFree(h->cnt_s); cudaFree(h->hbuf);
   cudaFree(h->yacc); cudaFree(h->dev_status); cudaFree(h->counters); cudaFree(h->syncbuf); cudaFree(h->trace);
-  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->cmask); cudaFree(h->umask);
+  cudaFree(h->u_in); cudaFree(h->u_ch); cudaFree(h->u_cnt); cudaFree(h->xu); cudaFree(h->member); cudaFree(h->hb); cudaFree(h->gacc); cudaFree(h->pacc); cudaFree(h->xh); cudaFree(h->tokfac); cudaFree(h->xd); cudaFree(h->soffb); cudaFree(h->cmask); cudaFree(h->umask);
   cudaFree(h->x_stage); cudaFree(h->y_stage);
   if (h->host_flag) cudaFreeHost(h->host_flag);
   if (h->prof) {
@@ -839,7 +905,7 @@ prox_status_t prox_stage1_mask(prox_ffn_t* h, const void* x, int B, int k1, int 
   const int D = h->cfg.d_model;
   float* sc = scores ? scores : h->scores;
   if (B > 1 && h->mask_policy == 1 && !(h->use_union && batch_path_ok(h, B, true))) return PROX_ERR_UNSUPPORTED;
-  if (h->use_union && batch_path_ok(h, B, true)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st);
+  if (h->use_union && batch_path_ok(h, B, true)) return launch_stage1_batch(h, x, B, k1, k2, sel, k2, sc, st, false, scores != nullptr);
   if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
   if ((s = launch_proxy(h, x, B, h->idx_x, D, nullptr, k1, sc, st)) != PROX_OK) return s;
   return launch_channel_select(h, sc, B, k2, 0.f, 0, sel, k2, nullptr, st);

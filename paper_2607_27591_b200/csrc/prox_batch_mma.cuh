@@ -628,18 +628,26 @@ proxy_mma_finish_kernel(float* __restrict__ pacc, int B, int F, float* __restric
 // tokfac[b] = 2^24 / s.  Token slots beyond B are cleared.
 __global__ void __launch_bounds__(kFusedThreads)
 batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __half* __restrict__ xh,
-                        float* __restrict__ tokfac) {
+                        float* __restrict__ tokfac, uint32_t* __restrict__ xd, float* __restrict__ soff) {
   extern __shared__ __align__(16) uint8_t bm_smem[];
   uint16_t* xs = reinterpret_cast<uint16_t*>(bm_smem);           // [D] bf16 bits of the token
   __shared__ unsigned hist[1024], hist2[32], wsum[32], smax;
+  __shared__ int sd[128 * 4];                                     // digit sums of the units of 128 inputs
   constexpr int NT = kFusedThreads;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the proxy GEMM may set up and start on the weights
   __half* row = xh + (size_t)b * D;
   if (b >= B) {
-    for (int i = tid; i < D / 8; i += NT) reinterpret_cast<uint4*>(row)[i] = make_uint4(0, 0, 0, 0);
+    if (xd) {
+      for (int i = tid; i < D; i += NT) xd[(size_t)(i >> 5) * 256 + (b >> 2) * 128 + (i & 31) * 4 + (b & 3)] = 0u;
+      for (int u = tid; u < (D >> 7); u += NT) soff[(size_t)u * kBT + b] = 0.f;
+    } else {
+      for (int i = tid; i < D / 8; i += NT) reinterpret_cast<uint4*>(row)[i] = make_uint4(0, 0, 0, 0);
+    }
     if (tid == 0) tokfac[b] = 16777216.f;
     return;
   }
+  for (int i = tid; i < 512; i += NT) sd[i] = 0;
   if (tid == 0) smax = 0;
   for (int i = tid; i < 1024 + 32; i += NT) { if (i < 1024) hist[i] = 0; else hist2[i - 1024] = 0; }
   __syncthreads();
@@ -707,6 +715,8 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
     const uint4 kv = *reinterpret_cast<const uint4*>(xs + g * 8);
     const uint32_t w4[4] = {kv.x, kv.y, kv.z, kv.w};
     uint32_t o[4];
+    int d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+    uint32_t* dst = xd ? xd + (size_t)(g >> 2) * 256 + (b >> 2) * 128 + ((g & 3) * 8) * 4 + (b & 3) : nullptr;
 #pragma unroll
     for (int e2 = 0; e2 < 4; ++e2) {
       __half hv[2];
@@ -717,10 +727,32 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
         const bool keep = gt || (eq && re < quota);
         re += eq ? 1u : 0u;
         hv[hh] = __float2half_rn(keep ? __uint_as_float(bits << 16) * sf : 0.f);
+        if (xd) {
+          // integer form of the masked, scaled fp16 input: X = x_h * 2^16 as four signed base-256 digits
+          const int X = __float2int_rn(__half2float(hv[hh]) * 65536.f);
+          const uint32_t dg = ((uint32_t)X + 0x00808080u) ^ 0x00808080u;
+          dst[(e2 * 2 + hh) * 4] = dg;
+          d0 += (int)(int8_t)(dg & 0xffu); d1 += (int)(int8_t)((dg >> 8) & 0xffu);
+          d2 += (int)(int8_t)((dg >> 16) & 0xffu); d3 += (int)(int8_t)(dg >> 24);
+        }
       }
       o[e2] = (uint32_t)__half_as_ushort(hv[0]) | ((uint32_t)__half_as_ushort(hv[1]) << 16);
     }
-    reinterpret_cast<uint4*>(row)[g] = make_uint4(o[0], o[1], o[2], o[3]);
+    if (xd) {
+      int* sdg = sd + 4 * (g >> 4);
+      if (d0) atomicAdd(sdg, d0);
+      if (d1) atomicAdd(sdg + 1, d1);
+      if (d2) atomicAdd(sdg + 2, d2);
+      if (d3) atomicAdd(sdg + 3, d3);
+    } else {
+      reinterpret_cast<uint4*>(row)[g] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+  if (xd) {
+    __syncthreads();
+    for (int u = tid; u < (D >> 7); u += NT)
+      soff[(size_t)u * kBT + b] = digits_to_float((uint32_t)sd[u * 4], (uint32_t)sd[u * 4 + 1], (uint32_t)sd[u * 4 + 2],
+                                                  (uint32_t)sd[u * 4 + 3]);
   }
 }
 
@@ -751,7 +783,7 @@ __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ s
 // over the summed scores) the kept channels get all of token_bits.
 __global__ void __launch_bounds__(kFusedThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
-                          unsigned* __restrict__ cmask, unsigned token_bits) {
+                          unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc) {
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
   __shared__ unsigned hist[2048], wsum[32], wsum2[32];
@@ -759,8 +791,21 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned* gkey = reinterpret_cast<const unsigned*>(scores) + (size_t)b * F;
   const uint32_t skey_u32 = smem_u32(skey);
-  for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
-  cp_async_commit();
+  if (pacc) {
+    // scores straight from the proxy sums of the tensor-core GEMM ([token][gate | up][channel]); the
+    // token's entries are cleared for the next call
+    float4* pg = reinterpret_cast<float4*>(pacc + (size_t)b * 2 * F);
+    float4* pu = pg + F / 4;
+    for (int i = tid; i < F / 4; i += NT) {
+      const float4 g = pg[i], u = pu[i];
+      pg[i] = make_float4(0.f, 0.f, 0.f, 0.f); pu[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      reinterpret_cast<uint4*>(skey)[i] = make_uint4(__float_as_uint(fabsf(u.x * silu_fast(g.x))), __float_as_uint(fabsf(u.y * silu_fast(g.y))),
+                                                     __float_as_uint(fabsf(u.z * silu_fast(g.z))), __float_as_uint(fabsf(u.w * silu_fast(g.w))));
+    }
+  } else {
+    for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
+    cp_async_commit();
+  }
   for (int i = tid; i < 2048; i += NT) hist[i] = 0;
   cp_async_wait<0>();
   __syncthreads();

@@ -822,11 +822,11 @@ def test_forms_on_odd_shapes(pb, D, F, bits, group):
         p.close()
 
 
-@pytest.mark.parametrize("group,B", [(0, 2), (128, 5), (128, 8)])
-def test_shared_batch_mask_policy(pb, toy, group, B):
+@pytest.mark.parametrize("bits,group,B", [(4, 0, 2), (4, 128, 5), (4, 128, 8), (8, 0, 8), (8, 128, 3)])
+def test_shared_batch_mask_policy(pb, toy, bits, group, B):
     """One channel mask for the batch, from the summed proxy scores; Stage 2 of every token on that mask."""
     wl, p = toy
-    dg, du, _ = p.quantize(4, group)
+    dg, du, _ = p.quantize(bits, group)
     k1, k2 = wl.points[50]
     t0 = 4
     pb.prox_ffn_set_mask_policy(p.h, 1)
@@ -852,8 +852,8 @@ def test_shared_batch_mask_policy(pb, toy, group, B):
         assert pb.prox_last_device_status(p.h) == 0
     finally:
         pb.prox_ffn_set_mask_policy(p.h, 0)
-    # 8-bit proxies do not have the tensor-core Stage 1: the policy is refused, not ignored
-    p.quantize(8, 0)
+    # 16-bit proxies do not have the tensor-core Stage 1: the policy is refused, not ignored
+    p.quantize(16, 0)
     pb.prox_ffn_set_mask_policy(p.h, 1)
     try:
         assert pb.raw("prox_ffn_forward")(p.h, p.t_x[:2].data_ptr(), 2, k1, k2, p.y_empty(2).data_ptr(), None) == 2
