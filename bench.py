@@ -54,8 +54,13 @@ def parse():
     ap.add_argument("--small-case", nargs="*", default=None, metavar="ARG",
                     help="profiler target instead of the benchmark: [workload] [calls] [batch] [topk|threshold|block]; two weight "
                          "replicas, a handful of launches, < 2 GB on the device")
-    ap.add_argument("--alpha", action="store_true",
-                    help="also measure the proxy-cost ratio alpha (integer proxy GEMV / 16-bit GEMV at equal input sparsity)")
+    ap.add_argument("--no-alpha", dest="alpha", action="store_false",
+                    help="skip the proxy-cost ratio alpha (integer proxy GEMV / 16-bit GEMV at equal input sparsity)")
+    ap.add_argument("--alpha", dest="alpha", action="store_true", help=argparse.SUPPRESS)   # measured by default
+    ap.add_argument("--rendezvous-only", action="store_true", help=argparse.SUPPRESS)   # CPU test of the N > 1 launch
+    ap.add_argument("--no-shapes", dest="shapes", action="store_false",
+                    help="skip the side measurements on the Llama-3-8B / Llama-3-70B shaped layers")
+    ap.set_defaults(alpha=True, shapes=True)
     return ap.parse_args()
 
 
@@ -409,6 +414,64 @@ def run_prox(args):
                   "masks": "per token; weights read once for the union",
                   "shared_mask_us_per_call": s8_us / calls8 if s8_us else None}
 
+        # The other layer shapes of the workload list, as side measurements: batch 1 and 8, every proxy format of
+        # the shape, and the ten-point sweep of the Stage-1 budget on the widest layer (two weight replicas per
+        # shape, every call on the other one: cold HBM).  Same call, same launch form (graph replay) as above.
+        shapes, s1_sweep = None, None
+        if args.shapes and rank == 0 and world == 1:
+            try:
+                shapes, s1_sweep = [], []
+                peak_gbs = peaks()[0]
+                for name in ("llama3_8b", "llama3_70b"):
+                    w2 = inputs.WORKLOADS[name]
+                    D2, F2 = w2.d_model, w2.d_ff
+                    reps2 = [tuple((torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * w2.w_std).to(torch.bfloat16)
+                                   for shape in ((F2, D2), (F2, D2), (D2, F2))) for _ in range(2)]
+                    hs2 = [pb.prox_ffn_create(D2, F2, 8, 0, *w) for w in reps2]
+                    xs2 = torch.from_numpy(np.ascontiguousarray(inputs.make_tokens(
+                        64, D2, w2.outlier_frac, w2.outlier_gain, w2.outlier_fixed_channels,
+                        np.random.default_rng(7))).view(np.int16)).to(dev).view(torch.bfloat16)
+                    ys2 = torch.empty(64, D2, dtype=torch.bfloat16, device=dev)
+
+                    def time_point(B2, k1b, k2b):
+                        def step():
+                            cs = torch.cuda.current_stream().cuda_stream
+                            for c in range(8):
+                                lo = (c * B2) % 64
+                                pb.prox_ffn_forward(hs2[c % 2], xs2[lo:lo + B2], B2, k1b, k2b, ys2[lo:lo + B2], stream=cs)
+                        us = timed_graph(step)
+                        return us / 8 if us else None
+
+                    for fmt in w2.proxies:
+                        for h in hs2:
+                            pb.prox_quantize_proxy(h, *fmt)
+                        torch.cuda.synchronize()
+                        for e_pct, (k1b, k2b) in sorted(w2.points.items()):
+                            for B2 in (1, 8):
+                                us = time_point(B2, k1b, k2b)
+                                row = {"workload": name, "d_model": D2, "d_ff": F2, "proxy": f"int{fmt[0]} group-{fmt[1]}",
+                                       "batch": B2, "e_pct": e_pct, "k1": k1b, "k2": k2b, "us_per_call": us}
+                                if B2 == 1 and us:
+                                    nb = sum(pb.prox_algorithmic_bytes(hs2[0], k1b, k2b))
+                                    row["algorithmic_bytes"] = nb
+                                    row["hbm_gbs"] = nb / us / 1e3
+                                    row["hbm_frac"] = nb / us / 1e3 / peak_gbs
+                                shapes.append(row)
+                        if "s1_sweep" in w2.extra and fmt == w2.proxies[-1]:
+                            for k1b, k2b in w2.extra["s1_sweep"]:
+                                us = time_point(1, k1b, k2b)
+                                nb = sum(pb.prox_algorithmic_bytes(hs2[0], k1b, k2b))
+                                s1_sweep.append({"workload": name, "proxy": f"int{fmt[0]} group-{fmt[1]}", "batch": 1,
+                                                 "k1": k1b, "k2": k2b, "us_per_call": us, "algorithmic_bytes": nb,
+                                                 "hbm_gbs": nb / us / 1e3 if us else None,
+                                                 "hbm_frac": nb / us / 1e3 / peak_gbs if us else None})
+                    for h in hs2:
+                        pb.prox_ffn_destroy(h)
+                    del reps2, hs2, xs2, ys2
+                    torch.cuda.empty_cache()
+            except Exception as ex:                    # pragma: no cover
+                sys.stderr.write(f"shape side measurements failed: {ex}\n")
+
         # The FFN sub-blocks of a 36-layer decoder applied to one residual stream, one graph per token
         # (RMSNorm + Prox FFN + residual add per layer in one launch each; layer l reads replica l mod R).
         LAYERS = 36
@@ -570,21 +633,29 @@ def run_prox(args):
     for name, (n, tot_ms) in prof.items():
         if n:
             us = tot_ms / n * 1e3
-            per_kernel[name] = {"us": us, "launches_per_call": n / T,
-                                "gbs": kernel_bytes.get(name, 0) / us / 1e3}
-    dom = max(per_kernel, key=lambda k: per_kernel[k]["us"] * per_kernel[k]["launches_per_call"]) if per_kernel else None
+            per_kernel[name] = {"us_event_bracketed": us, "launches_per_call": n / T,
+                                "gbs_event_bracketed": kernel_bytes.get(name, 0) / us / 1e3,
+                                "timing": "one CUDA event pair around every launch of one extra, ungraphed step: "
+                                          "includes the events' own cost and the launch gap"}
+    dom = max(per_kernel, key=lambda k: per_kernel[k]["us_event_bracketed"] * per_kernel[k]["launches_per_call"]) if per_kernel else None
     roof = None
     if dom:
-        ach = per_kernel[dom]["gbs"]
+        ach = per_kernel[dom]["gbs_event_bracketed"]
         timing = "per-kernel CUDA events over one extra step"
         if dom == "prox_fused" and abs(launches_per_call - 1.0) < 1e-9:
             # the timed region is nothing but back-to-back launches of this kernel, one per call:
             # its average launch duration there (gaps included) is the step time over the calls
             ach = kernel_bytes[dom] / (ms / args.steps / T * 1e3) / 1e3
             timing = "CUDA events around the timed region / launches in it"
+            per_kernel[dom]["us"] = ms / args.steps / T * 1e3
+            per_kernel[dom]["gbs"] = ach
         roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s",
                 "frac": ach / peak, "peak_kind": peak_kind, "timing": timing,
                 "traffic": ncu_traffic() if dom == "prox_fused" else None,
+                "traffic_source": ("profiles/prox_fused_kernel_qwen3_8b_ncu_full.md: dram__bytes_read.sum + "
+                                   "dram__bytes_write.sum per launch, ncu capture of `python bench.py --small-case` "
+                                   "(same kernel, shape and budget as this workload, two weight replicas)")
+                if dom == "prox_fused" else None,
                 "bytes_per_launch": kernel_bytes.get(dom)}
 
     cpu = None
@@ -624,6 +695,8 @@ def run_prox(args):
             "gpu_launches": int(round(launches_per_call * T * args.steps)),
             "dense_cublas_bf16_us_per_call": dense_us,
             "batch8": batch8,
+            "shapes": shapes,
+            "s1_sweep": s1_sweep,
             "decode_stack": decode_stack,
             "threshold_mode": threshold_mode,
             "alpha": alpha,
@@ -687,10 +760,51 @@ def run_small_case(argv):
     sys.exit(0 if not any(status) else 1)
 
 
+def replica_launch_command(n: int, argv, port: int):
+    """The command that starts n single-GPU replica processes of this script on this node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def run_rendezvous_only(args):
+    """Test hook (no GPU): the ranks meet over gloo, exchange the timing scalars as the real run does and
+    rank 0 prints the JSON line's multi-rank fields."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    ms = max_over_ranks([10.0 + 5.0 * rank])[0]
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "n_gpus": world, "steps": args.steps, "ms_per_step": ms / args.steps,
+                          "value": whole_job_us_per_call(ms, world, args.steps, args.tokens), "unit": UNIT,
+                          "scaling": "weak", "rendezvous_only": True}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse()
     if args.small_case is not None:
         run_small_case(args.small_case)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: start the N replica processes here (one rank per GPU) and pass their
+        # output and exit code through
+        import subprocess
+        sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:], free_port())))
+    if args.rendezvous_only:
+        run_rendezvous_only(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -25,7 +25,11 @@ paper; the paper's closed forms q_Lap, q_G, eta, Corr; the residual bound
 invariants; a hand-worked 4x4 example; the ablation forms against the dense FFN
 (all inputs and channels kept, original weights as proxy) and against Stage 2 on
 the exact top-k of |s|; RMSNorm against the library's rms_norm and the layer
-block against its parts.  The mask and output *values* on random
+block against its parts; the calibration helpers: the counter-based generator
+against the published splitmix64 outputs, the quantile against the library's
+quantile routine and an arithmetic progression, the reservoir against its size /
+membership / uniformity properties, Alg. 1 against the realised sparsities of
+the calibration stream and its one-layer special case.  The mask and output *values* on random
 inputs have no worked example in the paper: parity unpinned for those beyond
 the properties above.
 """
@@ -39,6 +43,7 @@ __all__ = [
     "channel_threshold", "stage2", "forward", "forward_batch", "allocate_budget",
     "sparsity_to_k", "effective_sparsity", "proxy_values", "forward_proxy_values",
     "rmsnorm", "ffn_block", "ffn_stack", "forward_batch_shared",
+    "splitmix64_at", "reservoir", "empirical_quantile", "histogram_4096", "calibrate_stack",
 ]
 
 
@@ -324,3 +329,109 @@ def sparsity_to_k(s: float, dim: int) -> int:
     "retains the (1 - rho) d_ff coordinates" without a rounding rule."""
     k = int(np.floor((1.0 - s) * dim + 0.5))
     return max(1, min(dim, k))
+
+
+# ------------------------------------------------ threshold calibration (Alg. 1)
+# Appendix "Threshold Calibration and Runtime Sparsity": per layer and per signal a
+# reservoir of at most 200,000 activation samples, the threshold "directly from the
+# corresponding empirical quantile", a 4,096-bin histogram saved beside it, layers
+# calibrated in depth order on the stream that the finalized sparse layers produce.
+_M64 = (1 << 64) - 1
+
+
+def splitmix64_at(seed: int, i: int) -> int:
+    """Output number i (0-based) of the splitmix64 sequence started at `seed`: a
+    counter-based generator (the state before output i is seed + (i+1)*gamma), so
+    that the reservoir's draws are a function of (seed, sample number) alone."""
+    z = (seed + (i + 1) * 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def reservoir(values, cap: int, seed: int, state=None):
+    """Uniform reservoir sampling (Vitter's algorithm R) of the magnitudes |v|, in
+    float32: the first `cap` samples fill the reservoir; sample number i >= cap
+    draws j = splitmix64_at(seed, i) mod (i + 1) and replaces slot j if j < cap.
+    `state` = (list, samples seen so far) continues an earlier call.
+    The paper fixes the capacity (200,000) but not the sampling scheme: this is
+    the textbook one.  Returns (list of float32 magnitudes, samples seen)."""
+    res, seen = ([], 0) if state is None else (list(state[0]), int(state[1]))
+    for v in np.asarray(values, dtype=np.float32).ravel():
+        m = np.float32(abs(v))
+        if seen < cap:
+            res.append(m)
+        else:
+            j = splitmix64_at(seed, seen) % (seen + 1)
+            if j < cap:
+                res[j] = m
+        seen += 1
+    return res, seen
+
+
+def empirical_quantile(mags, s: float) -> np.float32:
+    """Empirical quantile of the samples at level s with linear interpolation
+    between order statistics (position s*(n-1); the definition numpy and torch use
+    by default; the paper says only "empirical quantile").  Keeping |z| >= tau then
+    drops a fraction of about s of the samples.  Computed in float64, returned as
+    the float32 the kernels compare with."""
+    a = sorted(float(v) for v in mags)
+    n = len(a)
+    if n == 0:
+        raise ValueError("no samples")
+    pos = float(s) * (n - 1)
+    lo = int(np.floor(pos))
+    hi = min(lo + 1, n - 1)
+    return np.float32(a[lo] + (pos - lo) * (a[hi] - a[lo]))
+
+
+def histogram_4096(mags):
+    """The saved analysis artifact: 4,096 equal bins over [0, max |v|] of the
+    reservoir; a sample equal to the maximum falls into the last bin.  The paper
+    fixes the bin count only; range and binning are this reading.
+    Returns (int64 counts [4096], upper edge as float32)."""
+    a = np.asarray(list(mags), dtype=np.float32)
+    hi = np.float32(a.max()) if a.size else np.float32(0.0)
+    counts = np.zeros(4096, dtype=np.int64)
+    for v in a:
+        b = 4095 if hi == 0 else min(4095, int(np.floor(float(v) / float(hi) * 4096.0)))
+        counts[b] += 1
+    return counts, hi
+
+
+def calibrate_stack(x_res_tokens, layers, eps: float, s1: float, s2: float, cap: int = 200000, seed: int = 0):
+    """Alg. 1 (sequential threshold calibration) on a stack of FFN sub-blocks:
+    for layer l = 1..L: the calibration tokens arrive through layers 1..l-1 under
+    their finalized threshold rules; collect the layer's FFN inputs x_l; choose
+    tau_x as the s1-quantile of |x_l| and build m_x; compute the proxy state
+    s~_l = u~ * SiLU(g~) with m_x and the quantized proxies; choose tau_s as the
+    s2-quantile of |s~_l|; the layer's rule is final.  Because the stream that
+    reaches layer l+1 is the one the finalized rules of layers 1..l produce, it
+    is advanced layer by layer instead of being recomputed from the start.
+    `layers` = list of (norm_w, deq_gate, deq_up, w_gate, w_up, w_down) as in
+    `ffn_stack`; the FFN input is bf16(RMSNorm(x_res) * w).
+    Returns a list of dicts per layer: tau_x, tau_s, s1_hat, s2_hat (realised on
+    the calibration tokens), hist_x, hist_s."""
+    xs = [np.asarray(x, dtype=np.float64) for x in x_res_tokens]
+    out = []
+    for li, (nw, dg, du, wg, wu, wd) in enumerate(layers):
+        xn = [bf16_to_f64(f64_to_bf16_bits(rmsnorm(x, nw, eps))) for x in xs]
+        rx, _ = reservoir(np.concatenate(xn), cap, seed + 2 * li)
+        tau_x = empirical_quantile(rx, s1)
+        idx = [input_threshold(x, tau_x) for x in xn]
+        sc = [proxy_scores(x, i, dg, du) for x, i in zip(xn, idx)]
+        rs, _ = reservoir(np.concatenate(sc), cap, seed + 2 * li + 1)
+        tau_s = empirical_quantile(rs, s2)
+        kept_in = sum(len(i) for i in idx)
+        kept_ch = 0
+        nxt = []
+        for x_res, x, s_l in zip(xs, xn, sc):
+            sel = channel_threshold(s_l, tau_s)
+            kept_ch += len(sel)
+            nxt.append(x_res + stage2(x, sel, wg, wu, wd)[0])
+        out.append({"tau_x": tau_x, "tau_s": tau_s,
+                    "s1_hat": 1.0 - kept_in / (len(xs) * len(xs[0])),
+                    "s2_hat": 1.0 - kept_ch / (len(xs) * len(sc[0])),
+                    "hist_x": histogram_4096(rx), "hist_s": histogram_4096(rs)})
+        xs = nxt
+    return out

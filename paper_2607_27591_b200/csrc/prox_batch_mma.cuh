@@ -431,38 +431,10 @@ down_mma_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, c
 namespace prox {
 
 // ----------------------------------------------------------------------------
-// Stage 1 for B > 1 on the tensor cores (4-bit proxies).
-//
-// A 4-bit code c in the low mantissa bits of an fp16 with a zero exponent field
-// is the subnormal c * 2^-24, exactly.  So two codes of one channel taken from
-// two input rows become an fp16 K-pair with one byte permute and no offset to
-// subtract:
-//   ev = row & 0x0f0f0f0f (even codes, one per byte), od = (row >> 4) & 0x0f0f0f0f
-//   pair(code 2m) = bytes (evA[m], 0, evB[m], 0)   (the zero bytes replicate the sign of evA[m])
-// The 2^-24 and the per-token power-of-two scale of x are undone when a group is
-// closed, and the offset binary (c = q + 8) is removed with one more MMA whose A
-// operand is the constant 8: the same sums, the same rounding.
-//
-// Tiles: M = 16 codes columns (row g of A = code 2j of the lane's 8 bytes, row
-// g+8 = code 2j+1), N = 8 tokens, K = 16 consecutive inputs.  A lane loads 8 bytes
-// of a row: the gate half (g even) or the up half (g odd) of chunk g / 2 of a
-// 64-byte strip.  A K-block never straddles a quantization group (128 inputs), so
-// a warp closes a group by scaling its accumulators.
+// Input preparation of Stage 1 for B > 1 (the GEMM itself is the tcgen05 kernel
+// of prox_batch_umma.cuh): the step-wise fallback for shapes whose input mask
+// does not fit the one-block-per-token kernel further down.
 // ----------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t kpair(uint32_t lo, uint32_t hi, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(lo), "r"(hi), "r"(sel));
-  return d;
-}
-
-__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                        uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 // One block per token slot.  The token's kept inputs (its ascending index list)
 // become an fp16 vector over ALL inputs: x * s at a kept input, 0 elsewhere, with
 // s the power of two that puts max |x| into [2^13, 2^14).  With eight tokens the
@@ -494,125 +466,6 @@ proxy_xprep_kernel(const uint16_t* __restrict__ x, const int* __restrict__ idx, 
       const float v = __uint_as_float(((uint32_t)x[(size_t)b * D + i]) << 16) * s;
       row[i] = __float2half_rn(v);
     }
-  }
-}
-
-__global__ void __launch_bounds__(kMmaThreads, 1)
-proxy_mma_kernel(const uint8_t* __restrict__ P, const __half* __restrict__ S, const __half* __restrict__ xh,
-                 const float* __restrict__ tokfac, int D, int F, int gshift, float* __restrict__ pacc) {
-  extern __shared__ __align__(16) uint8_t mm_smem[];
-  float* red = reinterpret_cast<float*>(mm_smem);               // [warps][128 code columns][8 tokens]
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int nkb = D / 16;                                       // K-blocks of 16 consecutive inputs
-  const int kbshift = (gshift >= 31) ? 31 : gshift - 4;         // K-block -> quantization group
-  const int nchunks = F / 16, nstrip = nchunks / 4;
-  const size_t row_bytes = (size_t)nchunks * 16;
-  const long long total = (long long)nstrip * nkb;
-  long long u = total * blockIdx.x / gridDim.x;
-  const long long u1 = total * (blockIdx.x + 1) / gridDim.x;
-  const float tf0 = tokfac[2 * t], tf1 = tokfac[2 * t + 1];
-  while (u < u1) {
-    const int strip = (int)(u / nkb), a = (int)(u - (long long)strip * nkb);
-    const int b = (int)min((long long)nkb, a + (u1 - u));
-    const int chunk = strip * 4 + (g >> 1), half = g & 1;
-    const uint8_t* src = P + (size_t)strip * 64 + (size_t)g * 8;
-    const int wa = a + (int)(((long long)(b - a) * warp) / kMmaWarps), wb = a + (int)(((long long)(b - a) * (warp + 1)) / kMmaWarps);
-    float tot[8][4], acc[8][4], corr[4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { tot[j][q] = 0.f; acc[j][q] = 0.f; }
-    corr[0] = corr[1] = corr[2] = corr[3] = 0.f;
-    int curg = -1;
-    uint4 s0 = make_uint4(0, 0, 0, 0), s1 = s0;               // scales of the open group (requested when it opened)
-    auto open_group = [&](int grp) {
-      const uint4* sp = reinterpret_cast<const uint4*>(S + (((size_t)grp * nchunks + chunk) * 2 + half) * 16);
-      s0 = __ldg(sp); s1 = __ldg(sp + 1);
-    };
-    auto flush = [&](int grp) {
-      if (grp < 0) return;
-      const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float2 sc = __half22float2(*reinterpret_cast<const __half2*>(&sw[j]));     // codes 2j, 2j+1
-        tot[j][0] = fmaf((acc[j][0] - corr[0]) * tf0, sc.x, tot[j][0]);
-        tot[j][1] = fmaf((acc[j][1] - corr[1]) * tf1, sc.x, tot[j][1]);
-        tot[j][2] = fmaf((acc[j][2] - corr[0]) * tf0, sc.y, tot[j][2]);
-        tot[j][3] = fmaf((acc[j][3] - corr[1]) * tf1, sc.y, tot[j][3]);
-        acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-      }
-      corr[0] = corr[1] = corr[2] = corr[3] = 0.f;
-    };
-    auto load_unit = [&](int kb, uint2 (&w)[4], uint2& xp) {
-      const uint8_t* r0 = src + (size_t)(kb * 16 + 2 * t) * row_bytes;
-      w[0] = __ldg(reinterpret_cast<const uint2*>(r0));
-      w[1] = __ldg(reinterpret_cast<const uint2*>(r0 + row_bytes));
-      w[2] = __ldg(reinterpret_cast<const uint2*>(r0 + 8 * row_bytes));
-      w[3] = __ldg(reinterpret_cast<const uint2*>(r0 + 9 * row_bytes));
-      const uint32_t* xr = reinterpret_cast<const uint32_t*>(xh + (size_t)g * D + kb * 16 + 2 * t);
-      xp.x = __ldg(xr); xp.y = __ldg(xr + 4);
-    };
-    auto mma_unit = [&](int kb, const uint2 (&w)[4], const uint2& xp) {
-      const int grp = kb >> kbshift;
-      if (grp != curg) { flush(curg); curg = grp; open_group(grp); }
-      const uint32_t R[4][2] = {{w[0].x, w[0].y}, {w[1].x, w[1].y}, {w[2].x, w[2].y}, {w[3].x, w[3].y}};
-      uint32_t ev[4][2], od[4][2];                             // even / odd codes of the four rows, one per byte
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int wi = 0; wi < 2; ++wi) { ev[r][wi] = R[r][wi] & 0x0f0f0f0fu; od[r][wi] = (R[r][wi] >> 4) & 0x0f0f0f0fu; }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int wi = j >> 2;
-        const uint32_t m = (uint32_t)(j & 3);
-        // bytes (rowA[m], 0, rowB[m], 0): the zero bytes replicate the sign of rowA[m], which is below 16
-        const uint32_t sel = ((8u | m) << 12) | ((4u + m) << 8) | ((8u | m) << 4) | m;
-        mma_f16(acc[j], kpair(ev[0][wi], ev[1][wi], sel), kpair(od[0][wi], od[1][wi], sel),
-                kpair(ev[2][wi], ev[3][wi], sel), kpair(od[2][wi], od[3][wi], sel), xp.x, xp.y);
-      }
-      mma_f16(corr, 0x00080008u, 0x00080008u, 0x00080008u, 0x00080008u, xp.x, xp.y);
-    };
-    for (int kb = wa; kb < wb; kb += 2) {
-      uint2 w0[4], w1[4], xp0, xp1;
-      const bool two = kb + 1 < wb;
-      load_unit(kb, w0, xp0);
-      if (two) load_unit(kb + 1, w1, xp1);
-      mma_unit(kb, w0, xp0);
-      if (two) mma_unit(kb + 1, w1, xp1);
-    }
-    flush(curg);
-    // the warps' partial sums meet in shared memory: [code column g * 16 + c][token]
-    float* mine = red + warp * 1024;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      mine[(g * 16 + 2 * j) * 8 + 2 * t] = tot[j][0];     mine[(g * 16 + 2 * j) * 8 + 2 * t + 1] = tot[j][1];
-      mine[(g * 16 + 2 * j + 1) * 8 + 2 * t] = tot[j][2]; mine[(g * 16 + 2 * j + 1) * 8 + 2 * t + 1] = tot[j][3];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int rep = 0; rep < 2; ++rep) {
-      const int e = tid + rep * kMmaThreads;
-      float s = 0.f;
-#pragma unroll
-      for (int w = 0; w < kMmaWarps; ++w) s += red[w * 1024 + e];
-      atomicAdd(pacc + (size_t)strip * 1024 + e, s);
-    }
-    __syncthreads();
-    u += b - a;
-  }
-}
-
-// score[b][ch] = |up~ * SiLU(gate~)| from the accumulated sums; the accumulator is cleared for the next call.
-__global__ void __launch_bounds__(256)
-proxy_mma_finish_kernel(float* __restrict__ pacc, int B, int F, float* __restrict__ scores) {
-  for (int i = blockIdx.x * 256 + threadIdx.x; i < kBT * F; i += gridDim.x * 256) {
-    const int ch = i / kBT, b = i % kBT;
-    const int chunk = ch >> 4, c = ch & 15, strip = chunk >> 2, m = chunk & 3;
-    float* pg = pacc + (size_t)strip * 1024 + (size_t)((2 * m) * 16 + c) * 8 + b;
-    float* pu = pacc + (size_t)strip * 1024 + (size_t)((2 * m + 1) * 16 + c) * 8 + b;
-    const float gate = *pg, up = *pu;
-    *pg = 0.f; *pu = 0.f;
-    if (b < B) scores[(size_t)b * F + ch] = fabsf(up * silu_fast(gate));
   }
 }
 

@@ -575,3 +575,118 @@ def test_shared_mask_batch_reduces_to_single_token_and_ignores_token_order():
         m[torch.from_numpy(sel3)] = 1.0
         np.testing.assert_allclose(ys3[b], (torch.from_numpy(wd) @ (s_full * m)).numpy(), rtol=1e-10, atol=1e-13)
         np.testing.assert_allclose(ysp[2 - b], ys3[b], rtol=0, atol=0)
+
+
+# ------------------------------------------------ threshold calibration (Alg. 1)
+def test_counter_based_generator_matches_published_splitmix64_outputs():
+    line = [l for l in open(os.path.join(GOLDEN, "closed_forms.txt")) if l.startswith("splitmix64 ")][0].split()
+    seed, want = int(line[1]), [int(v) for v in line[2:]]
+    assert [po.splitmix64_at(seed, i) for i in range(len(want))] == want
+
+
+def test_empirical_quantile_against_library_and_closed_form():
+    rng = np.random.default_rng(5)
+    for n in (1, 2, 7, 100, 1001):
+        a = np.abs(rng.standard_normal(n)).astype(np.float32)
+        for s in (0.0, 0.1, 0.5, 0.7, 0.767, 1.0):
+            got = po.empirical_quantile(a, s)
+            assert got.dtype == np.float32
+            assert got == np.float32(np.quantile(a.astype(np.float64), s))
+    # arithmetic progression 0, 1, ..., n-1: the s-quantile is s * (n - 1)
+    assert po.empirical_quantile(np.arange(11, dtype=np.float32), 0.7) == np.float32(7.0)
+    assert po.empirical_quantile(np.arange(5, dtype=np.float32), 0.6) == np.float32(2.4)
+    # keeping |z| >= tau drops about a fraction s
+    a = np.abs(rng.laplace(size=5000)).astype(np.float32)
+    for s in (0.1, 0.55, 0.7):
+        tau = po.empirical_quantile(a, s)
+        assert abs(np.mean(a < tau) - s) <= 1.0 / a.size
+
+
+def test_reservoir_size_membership_order_and_uniformity():
+    v = np.arange(1, 101, dtype=np.float32) * np.where(np.arange(100) % 2 == 0, 1, -1)
+    res, seen = po.reservoir(v, cap=200, seed=3)
+    assert seen == 100 and res == [np.float32(i) for i in range(1, 101)]       # fewer than cap: all, in order, as magnitudes
+    # more than cap: exactly cap kept, every kept value comes from the stream, continuing a call changes nothing
+    n, cap = 20000, 500
+    stream = np.arange(n, dtype=np.float32)
+    res, seen = po.reservoir(stream, cap, seed=11)
+    assert seen == n and len(res) == cap and set(res) <= set(stream.tolist())
+    part, st = po.reservoir(stream[:7000], cap, seed=11)
+    res2, _ = po.reservoir(stream[7000:], cap, seed=11, state=(part, st))
+    assert res2 == res
+    # hand-checked replacement rule on a tiny case: sample number i >= cap goes to slot u_i mod (i + 1) when that is < cap
+    small, _ = po.reservoir(np.arange(6, dtype=np.float32), cap=3, seed=1)
+    expect = [0.0, 1.0, 2.0]
+    for i in (3, 4, 5):
+        j = po.splitmix64_at(1, i) % (i + 1)
+        if j < 3:
+            expect[j] = float(i)
+    assert [float(x) for x in small] == expect
+    # uniform: every stream position is kept with probability cap / n (mean of kept positions ~ n / 2; the
+    # standard error of that mean is n / sqrt(12 cap) ~ 258)
+    assert abs(float(np.mean(res)) - n / 2) < 4 * n / math.sqrt(12 * cap)
+    early = sum(1 for x in res if x < n / 4)
+    assert abs(early - cap / 4) < 4 * math.sqrt(cap * 0.25 * 0.75)
+
+
+def test_histogram_4096_counts_everything_once():
+    rng = np.random.default_rng(2)
+    a = np.abs(rng.standard_normal(3000)).astype(np.float32)
+    counts, hi = po.histogram_4096(a)
+    assert counts.shape == (4096,) and counts.sum() == a.size and hi == a.max()
+    ref, _ = np.histogram(a.astype(np.float64), bins=4096, range=(0.0, float(hi)))
+    assert np.abs(counts - ref).sum() <= 4                  # bin edges in float32 vs float64: a few borderline samples
+    assert counts[-1] >= 1                                  # the maximum itself lands in the last bin
+    z, hz = po.histogram_4096(np.zeros(5, dtype=np.float32))
+    assert hz == 0 and z[-1] == 5
+
+
+def _toy_stack(n_layers=3, d_model=128, d_ff=256, n_tok=12, seed=9):
+    layers = []
+    for l in range(n_layers):
+        wg, wu, wd, x = inputs.make_small(d_model, d_ff, n_tok, seed + l, std=0.05)
+        wg, wu, wd = po.bf16_to_f64(wg), po.bf16_to_f64(wu), po.bf16_to_f64(wd)
+        qg, sg = po.quantize_proxy(wg, 4, 0)
+        qu, su = po.quantize_proxy(wu, 4, 0)
+        nw = 1.0 + 0.1 * np.cos(np.arange(d_model) + l)
+        layers.append((po.bf16_to_f64(po.f64_to_bf16_bits(nw)), po.dequantize(qg, sg, 0), po.dequantize(qu, su, 0), wg, wu, wd))
+    return layers, po.bf16_to_f64(x)
+
+
+def test_sequential_calibration_realises_its_targets_and_sees_the_sparse_stream():
+    """Alg. 1: thresholds are quantiles of the very samples they are then applied to, so on the calibration tokens
+    every layer realises (s1, s2) to within one sample; layer l's thresholds come from the stream that the
+    finalized rules of layers 1..l-1 produce, not from the dense stream."""
+    layers, x0 = _toy_stack()
+    s1, s2, eps = 0.55, 0.7, 1e-6
+    cal = po.calibrate_stack(x0, layers, eps, s1, s2)
+    n_tok, D, F = x0.shape[0], x0.shape[1], layers[0][3].shape[0]
+    for c in cal:
+        assert abs(c["s1_hat"] - s1) <= 4.0 / (n_tok * D) + 1e-12      # bf16 inputs: a few equal magnitudes at the threshold
+        assert abs(c["s2_hat"] - s2) <= 1.5 / (n_tok * F) + 1e-12
+        assert c["hist_x"][0].sum() == n_tok * D and c["hist_s"][0].sum() == n_tok * F
+    # one layer alone = plain quantiles of that layer's own signals, by library routines
+    nw, dg, du = layers[0][0], layers[0][1], layers[0][2]
+    xn = np.stack([po.bf16_to_f64(po.f64_to_bf16_bits(po.rmsnorm(x, nw, eps))) for x in x0])
+    tx = np.float32(np.quantile(np.abs(xn).astype(np.float32).astype(np.float64), s1))
+    assert cal[0]["tau_x"] == tx
+    sc = []
+    for x in xn:
+        xm = np.where(np.abs(x) >= tx, x, 0.0)
+        g, u = torch.from_numpy(dg) @ torch.from_numpy(xm), torch.from_numpy(du) @ torch.from_numpy(xm)
+        sc.append((u * torch.nn.functional.silu(g)).abs().numpy())
+    ts = np.float32(np.quantile(np.concatenate(sc).astype(np.float32).astype(np.float64), s2))
+    assert abs(float(cal[0]["tau_s"]) - float(ts)) <= 1e-6 * float(ts)
+    # the stream matters: layer 2 calibrated behind a dense layer 1 gets other thresholds
+    dense_first = po.calibrate_stack(x0, layers, eps, 0.0, 0.0)
+    later = po.calibrate_stack([po.ffn_stack(x, layers[:1], eps, D, F)[-1] for x in x0], layers[1:], eps, s1, s2)
+    assert dense_first[0]["s1_hat"] == 0.0 and dense_first[0]["s2_hat"] == 0.0
+    assert later[0]["tau_x"] != cal[1]["tau_x"] or later[0]["tau_s"] != cal[1]["tau_s"]
+    # ... and equals a calibration started from the sparse stream of layer 1 under its finalized rule
+    x1 = []
+    for x in x0:
+        x_in = po.bf16_to_f64(po.f64_to_bf16_bits(po.rmsnorm(x, nw, eps)))
+        sel = po.channel_threshold(po.proxy_scores(x_in, po.input_threshold(x_in, cal[0]["tau_x"]), dg, du), cal[0]["tau_s"])
+        x1.append(x + po.stage2(x_in, sel, layers[0][3], layers[0][4], layers[0][5])[0])
+    tail = po.calibrate_stack(x1, layers[1:], eps, s1, s2, seed=2)
+    assert tail[0]["tau_x"] == cal[1]["tau_x"] and tail[0]["tau_s"] == cal[1]["tau_s"]
