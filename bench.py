@@ -497,7 +497,15 @@ def run_prox(args):
         try:
             s1_t, s2_t = 1.0 - k1 / D, 1.0 - k2 / F
             ncal = 64
-            tau_x = float(torch.quantile(x[:ncal].float().abs().flatten(), s1_t))
+            def calib_quantile(values, dtype_code, level):
+                # the library's calibration state (reservoir of <= 200,000 magnitudes, empirical quantile)
+                c = pb.prox_calib_create(200000, 0)
+                try:
+                    pb.prox_calib_add(c, values, values.numel(), dtype_code, stream=sp)
+                    return pb.prox_calib_threshold(c, level)
+                finally:
+                    pb.prox_calib_destroy(c)
+            tau_x = calib_quantile(x[:ncal].contiguous(), 0, s1_t)
             sc = torch.empty(ncal, F, dtype=torch.float32, device=dev)
             selc = torch.empty(1, F, dtype=torch.int32, device=dev)
             cntc = torch.empty(1, dtype=torch.int32, device=dev)
@@ -506,7 +514,7 @@ def run_prox(args):
                 for i in range(ncal):
                     pb.prox_stage1_mask_threshold(handles[r], x[i], 1, tau_x, 0.0, selc, cntc, sc[i], stream=sp)
                 stream.synchronize()
-                tau_s.append(float(torch.quantile(sc.flatten(), s2_t)))
+                tau_s.append(calib_quantile(sc, 1, s2_t))
             for h in handles:
                 pb.prox_runtime_sparsity(h, reset=True)
 
@@ -526,28 +534,15 @@ def run_prox(args):
         except Exception as ex:                        # pragma: no cover
             sys.stderr.write(f"threshold-mode measurement failed: {ex}\n")
 
-        # The same 36-layer loop with thresholded masks (per-layer thresholds calibrated on the streams of
-        # the first tokens: tau_x over |FFN input| at level s1, tau_s over the proxy scores at level s2).
+        # The same 36-layer loop with thresholded masks: per-layer thresholds from the sequential calibration of
+        # Alg. 1 on the first tokens (tau_x over |FFN input| at level s1, tau_s over the proxy scores at level s2,
+        # every layer calibrated on the stream its finalized predecessors produce).
         try:
             ncal = 8
             s1_t, s2_t = 1.0 - k1 / D, 1.0 - k2 / F
-            tr = torch.empty(ncal, LAYERS + 1, D, dtype=torch.float32, device=dev)
-            for i in range(ncal):
-                xi = x[i:i + 1].float().contiguous()
-                pb.prox_ffn_stack_forward(stack_handles, nw, 1e-6, xi, 1, k1, k2, tr[i], stream=sp)
-            stream.synchronize()
-            ltx, lts = [], []
-            scl = torch.empty(ncal, F, dtype=torch.float32, device=dev)
-            sel_l = torch.empty(1, F, dtype=torch.int32, device=dev)
-            cnt_l = torch.empty(1, dtype=torch.int32, device=dev)
-            for l in range(LAYERS):
-                xin = tr[:, l, :]
-                xn = (xin * torch.rsqrt((xin * xin).mean(dim=1, keepdim=True) + 1e-6) * nw[l].float()).to(torch.bfloat16)
-                ltx.append(float(torch.quantile(xn.float().abs().flatten(), s1_t)))
-                for i in range(ncal):
-                    pb.prox_stage1_mask_threshold(stack_handles[l], xn[i], 1, ltx[-1], 0.0, sel_l, cnt_l, scl[i], stream=sp)
-                stream.synchronize()
-                lts.append(float(torch.quantile(scl.flatten(), s2_t)))
+            # sequential calibration (Alg. 1) through the library: layer after layer on the sparse stream
+            ltx, lts, _ = pb.prox_calibrate_stack(stack_handles, F, nw, 1e-6, x[:ncal].float().contiguous(), s1_t, s2_t,
+                                                  stream=sp)
             for h in handles:
                 pb.prox_runtime_sparsity(h, reset=True)
 

@@ -302,6 +302,36 @@ prox_status_t prox_ffn_stack_forward_threshold(prox_ffn_t* const* layers, int n_
                                                double eps, float* x_res_dev, int B, const float* tau_x_host,
                                                const float* tau_s_host, float* trace_dev_or_null, void* stream);
 
+/* ---- Offline threshold calibration (appendix "Threshold Calibration and Runtime Sparsity", Alg. 1).
+ * Host-side state of one (layer, signal) pair: a reservoir of at most `capacity` activation magnitudes
+ * (the paper keeps at most 200,000), the threshold "directly from the corresponding empirical quantile",
+ * and the saved 4,096-bin histogram.  Not part of the decode hot path: the calls synchronise.
+ * Sampling: uniform reservoir (algorithm R); sample number i >= capacity draws
+ * j = splitmix64(seed; output i) mod (i + 1) and replaces slot j if j < capacity, so the result is a
+ * function of (seed, order of the samples) alone.
+ *   prox_calib_add        values_dev: dev bf16 (dtype 0) or fp32 (dtype 1) [n]; |v| is stored as fp32.
+ *   prox_calib_threshold  the s-quantile of the reservoir, linear interpolation between order statistics
+ *                         (position s (n - 1)), computed in double, returned as the fp32 the kernels
+ *                         compare with (|x_i| >= tau_x, score_j >= tau_s).
+ *   prox_calib_histogram  counts_host: int64 [4096], equal bins over [0, max]; upper = max magnitude.
+ *   prox_calib_seen       samples offered so far / samples held.
+ * Errors: INVALID_ARG (NULL, capacity < 1, s outside [0, 1], dtype), NOT_QUANTIZED is not involved,
+ * UNSUPPORTED (threshold or histogram of an empty reservoir), CUDA, OOM. */
+typedef struct prox_calib prox_calib_t;
+prox_status_t prox_calib_create(int64_t capacity, uint64_t seed, prox_calib_t** out);
+void prox_calib_destroy(prox_calib_t* c);
+prox_status_t prox_calib_add(prox_calib_t* c, const void* values_dev, int64_t n, int dtype, void* stream);
+prox_status_t prox_calib_threshold(const prox_calib_t* c, double s, float* tau);
+prox_status_t prox_calib_histogram(const prox_calib_t* c, int64_t* counts_host, float* upper);
+prox_status_t prox_calib_seen(const prox_calib_t* c, int64_t* seen, int64_t* held);
+
+/* The FFN input of a layer as the block calls form it: xn = bf16(RMSNorm(x_res) * w)
+ * (x_res dev fp32 [B, d_model], norm_w dev bf16 [d_model], xn_out dev bf16 [B, d_model]).  Alg. 1
+ * collects these as the layer's calibration inputs.  Enqueued on stream.
+ * Errors: INVALID_ARG, UNSUPPORTED (B > max_batch), CUDA. */
+prox_status_t prox_rmsnorm(prox_ffn_t* h, const float* x_res_dev, const void* norm_w_dev, double eps, int B,
+                           void* xn_out_dev, void* stream);
+
 /* Runtime mask counts accumulated by the threshold entry points since the last
  * reset (appendix "Threshold Calibration and Runtime Sparsity":
  * e^ = s2^ - 2 alpha (1 - s1^) / 3).  Host-synchronous.  Any pointer may be NULL. */

@@ -76,6 +76,12 @@ _SIGS = {
     "prox_ffn_last_mask": [_vp, _i, _i, _vp, _vp],
     "prox_ffn_last_stage1": [_vp, _i, _vp, _vp, _vp],
     "prox_debug_set_wait": [_vp, C.c_uint32, C.c_uint32],
+    "prox_calib_create": [C.c_int64, C.c_uint64, C.POINTER(_vp)],
+    "prox_calib_add": [_vp, _vp, C.c_int64, _i, _vp],
+    "prox_calib_threshold": [_vp, _d, C.POINTER(_f)],
+    "prox_calib_histogram": [_vp, C.POINTER(C.c_int64), C.POINTER(_f)],
+    "prox_calib_seen": [_vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
+    "prox_rmsnorm": [_vp, _vp, _vp, _d, _i, _vp, _vp],
     "prox_profile_enable": [_vp, _i],
     "prox_profile_read": [_vp, C.POINTER(C.c_int64), C.POINTER(_d)],
 }
@@ -85,6 +91,8 @@ for _name, _args in _SIGS.items():
     _fn.restype = C.c_int
 _lib.prox_ffn_destroy.argtypes = [_vp]
 _lib.prox_ffn_destroy.restype = None
+_lib.prox_calib_destroy.argtypes = [_vp]
+_lib.prox_calib_destroy.restype = None
 _lib.prox_status_string.argtypes = [C.c_int]
 _lib.prox_status_string.restype = C.c_char_p
 _lib.prox_last_cuda_error.argtypes = []
@@ -92,7 +100,7 @@ _lib.prox_last_cuda_error.restype = C.c_char_p
 _lib.prox_version.argtypes = []
 _lib.prox_version.restype = C.c_char_p
 
-EXPORTED = tuple(_SIGS) + ("prox_ffn_destroy", "prox_status_string", "prox_version", "prox_last_cuda_error")
+EXPORTED = tuple(_SIGS) + ("prox_ffn_destroy", "prox_calib_destroy", "prox_status_string", "prox_version", "prox_last_cuda_error")
 
 
 def _ptr(obj) -> Optional[int]:
@@ -241,6 +249,86 @@ def prox_ffn_stack_forward_threshold(handles, norm_w, eps: float, x_res, B: int,
     ts = (_f * n)(*[float(v) for v in tau_s])
     _check(_lib.prox_ffn_stack_forward_threshold(arr, n, _ptr(norm_w), eps, _ptr(x_res), B, tx, ts, _ptr(trace),
                                                  _ptr(stream)), "prox_ffn_stack_forward_threshold")
+
+
+def prox_calib_create(capacity: int = 200000, seed: int = 0) -> int:
+    out = _vp()
+    _check(_lib.prox_calib_create(capacity, seed, C.byref(out)), "prox_calib_create")
+    return out.value
+
+
+def prox_calib_destroy(calib: int) -> None:
+    _lib.prox_calib_destroy(calib)
+
+
+def prox_calib_add(calib: int, values, n: int, dtype: int, stream=None) -> None:
+    """dtype 0: dev bf16 values, 1: dev fp32 values."""
+    _check(_lib.prox_calib_add(calib, _ptr(values), n, dtype, _ptr(stream)), "prox_calib_add")
+
+
+def prox_calib_threshold(calib: int, s: float) -> float:
+    tau = _f()
+    _check(_lib.prox_calib_threshold(calib, s, C.byref(tau)), "prox_calib_threshold")
+    return tau.value
+
+
+def prox_calib_histogram(calib: int):
+    counts = (C.c_int64 * 4096)()
+    hi = _f()
+    _check(_lib.prox_calib_histogram(calib, counts, C.byref(hi)), "prox_calib_histogram")
+    return list(counts), hi.value
+
+
+def prox_calib_seen(calib: int):
+    seen, held = C.c_int64(), C.c_int64()
+    _check(_lib.prox_calib_seen(calib, C.byref(seen), C.byref(held)), "prox_calib_seen")
+    return seen.value, held.value
+
+
+def prox_rmsnorm(handle: int, x_res, norm_w, eps: float, B: int, xn_out, stream=None) -> None:
+    _check(_lib.prox_rmsnorm(handle, _ptr(x_res), _ptr(norm_w), eps, B, _ptr(xn_out), _ptr(stream)), "prox_rmsnorm")
+
+
+def prox_calibrate_stack(handles, d_ff: int, norm_w, eps: float, x_res_tokens, s1: float, s2: float,
+                         capacity: int = 200000, seed: int = 0, stream=None):
+    """Sequential threshold calibration (Alg. 1) of a stack of FFN sub-blocks, driven through the library:
+    per layer, in depth order, on the stream that the finalized rules of the earlier layers produce:
+    FFN inputs (prox_rmsnorm) -> tau_x (reservoir quantile at s1) -> proxy scores under that input mask
+    (prox_stage1_mask_threshold) -> tau_s (quantile at s2) -> the tokens advance through the layer under
+    its finalized rule (prox_ffn_block_forward_threshold).
+    handles: one per layer (all of width d_ff); norm_w: dev bf16 [L, d_model]; x_res_tokens: dev fp32 [N, d_model] (left untouched).
+    Device buffers come from torch (plumbing); every step of the path is a library call.
+    Returns (tau_x list, tau_s list, list of (hist_x, hist_s) with hist = (counts[4096], upper edge))."""
+    import torch
+    N, D = x_res_tokens.shape
+    xs = x_res_tokens.clone()
+    nxt = torch.empty_like(xs)
+    dev = xs.device
+    xn = torch.empty(N, D, dtype=torch.bfloat16, device=dev)
+    sc = torch.empty(N, d_ff, dtype=torch.float32, device=dev)
+    sel = torch.empty(1, d_ff, dtype=torch.int32, device=dev)
+    cnt = torch.empty(1, dtype=torch.int32, device=dev)
+    tau_x, tau_s, hists = [], [], []
+    for li, h in enumerate(handles):
+        cx, cs = prox_calib_create(capacity, seed + 2 * li), prox_calib_create(capacity, seed + 2 * li + 1)
+        try:
+            for i in range(N):
+                prox_rmsnorm(h, xs[i], norm_w[li], eps, 1, xn[i], stream)
+            prox_calib_add(cx, xn, N * D, 0, stream)
+            tx = prox_calib_threshold(cx, s1)
+            for i in range(N):
+                prox_stage1_mask_threshold(h, xn[i], 1, tx, 0.0, sel, cnt, sc[i], stream)
+            prox_calib_add(cs, sc, sc.numel(), 1, stream)
+            ts = prox_calib_threshold(cs, s2)
+            for i in range(N):
+                prox_ffn_block_forward_threshold(h, xs[i], norm_w[li], eps, 1, tx, ts, nxt[i], stream)
+            hists.append((prox_calib_histogram(cx), prox_calib_histogram(cs)))
+        finally:
+            prox_calib_destroy(cx); prox_calib_destroy(cs)
+        tau_x.append(tx); tau_s.append(ts)
+        xs, nxt = nxt, xs
+    torch.cuda.synchronize(dev)
+    return tau_x, tau_s, hists
 
 
 def prox_runtime_sparsity(handle: int, alpha: float = 1.0 / 3.0, reset: bool = False):

@@ -2,6 +2,7 @@
 // Declarations and per-call documentation live in include/prox.h.
 #include "prox.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -1092,6 +1093,113 @@ prox_status_t prox_fused_trace(prox_ffn_t* h, int on, uint64_t* stamps_host, int
     CK(cudaMemcpy(stamps_host, h->trace, (size_t)n * 32 * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
   }
   if (!on && h->trace) { cudaFree(h->trace); h->trace = nullptr; }
+  return PROX_OK;
+}
+
+// ---- offline threshold calibration (host side) ---------------------------------
+struct prox_calib {
+  int64_t cap, seen;
+  uint64_t seed;
+  std::vector<float> res;
+  std::vector<char> stage;
+};
+
+static inline uint64_t splitmix64_at(uint64_t seed, uint64_t i) {
+  uint64_t z = seed + (i + 1) * 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+prox_status_t prox_calib_create(int64_t capacity, uint64_t seed, prox_calib_t** out) {
+  if (!out || capacity < 1 || capacity > (int64_t)1 << 28) return PROX_ERR_INVALID_ARG;
+  prox_calib* c = new (std::nothrow) prox_calib();
+  if (!c) return PROX_ERR_OOM;
+  c->cap = capacity; c->seen = 0; c->seed = seed;
+  *out = c;
+  return PROX_OK;
+}
+
+void prox_calib_destroy(prox_calib_t* c) { delete c; }
+
+prox_status_t prox_calib_add(prox_calib_t* c, const void* values_dev, int64_t n, int dtype, void* stream) {
+  if (!c || n < 0 || (n > 0 && !values_dev) || (dtype != 0 && dtype != 1)) return PROX_ERR_INVALID_ARG;
+  if (n == 0) return PROX_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t esz = dtype == 0 ? 2 : 4;
+  try { c->stage.resize((size_t)n * esz); } catch (...) { return PROX_ERR_OOM; }
+  CK(cudaMemcpyAsync(c->stage.data(), values_dev, (size_t)n * esz, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  try {
+    for (int64_t k = 0; k < n; ++k) {
+      float v;
+      if (dtype == 0) {
+        const uint32_t bits = (uint32_t)reinterpret_cast<const uint16_t*>(c->stage.data())[k] << 16;
+        std::memcpy(&v, &bits, 4);
+      } else {
+        v = reinterpret_cast<const float*>(c->stage.data())[k];
+      }
+      v = std::fabs(v);
+      if (c->seen < c->cap) {
+        c->res.push_back(v);
+      } else {
+        const uint64_t j = splitmix64_at(c->seed, (uint64_t)c->seen) % ((uint64_t)c->seen + 1);
+        if (j < (uint64_t)c->cap) c->res[(size_t)j] = v;
+      }
+      c->seen++;
+    }
+  } catch (...) { return PROX_ERR_OOM; }
+  return PROX_OK;
+}
+
+prox_status_t prox_calib_threshold(const prox_calib_t* c, double s, float* tau) {
+  if (!c || !tau || !(s >= 0.0 && s <= 1.0)) return PROX_ERR_INVALID_ARG;
+  if (c->res.empty()) return PROX_ERR_UNSUPPORTED;
+  std::vector<float> a;
+  try { a = c->res; } catch (...) { return PROX_ERR_OOM; }
+  std::sort(a.begin(), a.end());
+  const size_t n = a.size();
+  const double pos = s * (double)(n - 1);
+  const size_t lo = (size_t)std::floor(pos), hi = lo + 1 < n ? lo + 1 : n - 1;
+  *tau = (float)((double)a[lo] + (pos - (double)lo) * ((double)a[hi] - (double)a[lo]));
+  return PROX_OK;
+}
+
+prox_status_t prox_calib_histogram(const prox_calib_t* c, int64_t* counts_host, float* upper) {
+  if (!c || !counts_host || !upper) return PROX_ERR_INVALID_ARG;
+  if (c->res.empty()) return PROX_ERR_UNSUPPORTED;
+  float hi = 0.f;
+  for (float v : c->res) hi = v > hi ? v : hi;
+  for (int b = 0; b < 4096; ++b) counts_host[b] = 0;
+  for (float v : c->res) {
+    int b = 4095;
+    if (hi > 0.f) {
+      const double q = std::floor((double)v / (double)hi * 4096.0);
+      b = q < 4095.0 ? (int)q : 4095;
+    }
+    counts_host[b]++;
+  }
+  *upper = hi;
+  return PROX_OK;
+}
+
+prox_status_t prox_calib_seen(const prox_calib_t* c, int64_t* seen, int64_t* held) {
+  if (!c) return PROX_ERR_INVALID_ARG;
+  if (seen) *seen = c->seen;
+  if (held) *held = (int64_t)c->res.size();
+  return PROX_OK;
+}
+
+prox_status_t prox_rmsnorm(prox_ffn_t* h, const float* x_res, const void* norm_w, double eps, int B, void* xn_out,
+                           void* stream) {
+  prox_status_t s = check_common(h, x_res, B);
+  if (s != PROX_OK) return s;
+  if (!norm_w || !xn_out || !aligned16(xn_out) || !aligned16(norm_w) || !(eps >= 0.0)) return PROX_ERR_INVALID_ARG;
+  const int D = h->cfg.d_model;
+  rmsnorm_kernel<<<B, 256, 0, static_cast<cudaStream_t>(stream)>>>(x_res, static_cast<const uint16_t*>(norm_w), rms_const(D, eps), D,
+                                                                   static_cast<uint16_t*>(xn_out));
+  h->launches++;
+  CK(cudaGetLastError());
   return PROX_OK;
 }
 

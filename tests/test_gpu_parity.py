@@ -822,6 +822,90 @@ def test_forms_on_odd_shapes(pb, D, F, bits, group):
         p.close()
 
 
+def test_calibration_state_matches_the_oracle(pb):
+    """Reservoir, quantile and histogram of the library (host side, fed from device buffers) against the oracle's,
+    value for value: below and above the capacity, bf16 and fp32 samples, in two pieces."""
+    rng = np.random.default_rng(12)
+    v32 = rng.standard_normal(5000).astype(np.float32) * 3
+    bits = po.f64_to_bf16_bits(rng.laplace(size=3000))
+    from tests.gpu_common import dev_bf16
+    t32, t16 = torch.from_numpy(v32).cuda(), dev_bf16(bits)
+    for cap in (100000, 700):
+        c = pb.prox_calib_create(cap, 5)
+        try:
+            pb.prox_calib_add(c, t32[:1234], 1234, 1)
+            pb.prox_calib_add(c, t32[1234:], 5000 - 1234, 1)
+            pb.prox_calib_add(c, t16, 3000, 0)
+            res, seen = po.reservoir(v32, cap, 5)
+            res, seen = po.reservoir(po.bf16_to_f64(bits), cap, 5, state=(res, seen))
+            assert pb.prox_calib_seen(c) == (8000, min(cap, 8000))
+            for s_ in (0.0, 0.1, 0.55, 0.7, 0.767, 1.0):
+                assert np.float32(pb.prox_calib_threshold(c, s_)) == po.empirical_quantile(res, s_)
+            counts, hi = pb.prox_calib_histogram(c)
+            ref_counts, ref_hi = po.histogram_4096(res)
+            assert np.float32(hi) == ref_hi and np.array_equal(np.asarray(counts), ref_counts)
+        finally:
+            pb.prox_calib_destroy(c)
+    # error paths: empty reservoir, bad level
+    c = pb.prox_calib_create(10, 0)
+    try:
+        tau = pb._f()
+        assert pb.raw("prox_calib_threshold")(c, 0.5, tau) == 2            # UNSUPPORTED: nothing sampled
+        pb.prox_calib_add(c, t32, 5, 1)
+        assert pb.raw("prox_calib_threshold")(c, 1.5, tau) == 1            # INVALID_ARG
+    finally:
+        pb.prox_calib_destroy(c)
+
+
+def test_sequential_threshold_calibration_of_a_stack(pb):
+    """Alg. 1 through the library (RMSNorm -> tau_x -> proxy scores -> tau_s -> advance under the finalized
+    rule, layer after layer) against the oracle's calibrate_stack on the same tokens.  Layer 0 sees the same
+    inputs on both sides; later layers see streams that may differ where a score sits inside the threshold band,
+    so their thresholds are compared with a tolerance and through the sparsities they realise on the GPU's stream."""
+    from tests.gpu_common import dev_bf16
+    L, D, F, N = 3, 512, 1536, 12
+    probs = []
+    try:
+        for l in range(L):
+            wg, wu, wd, x = inputs.make_small(D, F, N, seed=80 + l)
+            probs.append(Problem(pb, wg, wu, wd, x, max_batch=1))
+        deqs = [q.quantize(4, 128) for q in probs]
+        nw_bits = np.stack([_norm_weight(D, 90 + l) for l in range(L)])
+        nw64 = [po.bf16_to_f64(nw_bits[l]) for l in range(L)]
+        t_nw = dev_bf16(nw_bits)
+        eps, s1, s2 = 1e-6, 0.55, 0.7
+        x0 = (probs[0].x[:N] * 2.0).astype(np.float32)
+        t_x = torch.from_numpy(x0).cuda()
+        tau_x, tau_s, hists = pb.prox_calibrate_stack([q.h for q in probs], F, t_nw, eps, t_x, s1, s2)
+        assert torch.equal(t_x.cpu(), torch.from_numpy(x0))
+        layers = [(nw64[l], deqs[l][0], deqs[l][1], probs[l].wg, probs[l].wu, probs[l].wd) for l in range(L)]
+        cal = po.calibrate_stack(x0.astype(np.float64), layers, eps, s1, s2)
+        # layer 0: the FFN inputs are bf16 values; the fp32 RMSNorm may round a handful of them to the neighbour
+        assert abs(tau_x[0] - float(cal[0]["tau_x"])) <= 2.0 ** -7 * float(cal[0]["tau_x"])
+        assert abs(tau_s[0] - float(cal[0]["tau_s"])) <= 2e-3 * float(cal[0]["tau_s"])
+        for l in range(L):
+            assert abs(tau_x[l] - float(cal[l]["tau_x"])) <= 0.02 * float(cal[l]["tau_x"])
+            assert abs(tau_s[l] - float(cal[l]["tau_s"])) <= 0.05 * float(cal[l]["tau_s"])
+            (cx, hx), (cs, hs) = hists[l]
+            assert sum(cx) == N * D and sum(cs) == N * F and hx > 0 and hs > 0
+        # the thresholds realise their targets on the calibration tokens when the stack then runs with them
+        for q in probs:
+            pb.prox_runtime_sparsity(q.h, reset=True)
+        for i in range(N):
+            xi = t_x[i:i + 1].clone()
+            pb.prox_ffn_stack_forward_threshold([q.h for q in probs], t_nw, eps, xi, 1, tau_x, tau_s)
+        torch.cuda.synchronize()
+        for q in probs:
+            tok, s1h, s2h, _ = pb.prox_runtime_sparsity(q.h)
+            assert tok == N
+            # bf16 inputs: about ten samples share the magnitude at the threshold (spacing 2^-8 of the value)
+            assert abs(s1h - s1) <= 24.0 / (N * D) + 1e-9 and abs(s2h - s2) <= 3.0 / (N * F) + 1e-9
+            assert pb.prox_last_device_status(q.h) == 0
+    finally:
+        for q in probs:
+            q.close()
+
+
 @pytest.mark.parametrize("bits,group,B", [(4, 0, 2), (4, 128, 5), (4, 128, 8), (8, 0, 8), (8, 128, 3)])
 def test_shared_batch_mask_policy(pb, toy, bits, group, B):
     """One channel mask for the batch, from the summed proxy scores; Stage 2 of every token on that mask."""

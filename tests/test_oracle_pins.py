@@ -579,7 +579,7 @@ def test_shared_mask_batch_reduces_to_single_token_and_ignores_token_order():
 
 # ------------------------------------------------ threshold calibration (Alg. 1)
 def test_counter_based_generator_matches_published_splitmix64_outputs():
-    line = [l for l in open(os.path.join(GOLDEN, "closed_forms.txt")) if l.startswith("splitmix64 ")][0].split()
+    line = [l for l in open(os.path.join(GOLDEN, "splitmix64_reference.txt")) if l.startswith("splitmix64 ")][0].split()
     seed, want = int(line[1]), [int(v) for v in line[2:]]
     assert [po.splitmix64_at(seed, i) for i in range(len(want))] == want
 
