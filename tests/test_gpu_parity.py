@@ -822,6 +822,28 @@ def test_forms_on_odd_shapes(pb, D, F, bits, group):
         p.close()
 
 
+def test_dff_shard_over_the_library_with_one_rank(pb, toy):
+    """The d_ff-sharded form with a single rank (no process group): the library's scores -> the exchange's global
+    top-k2 -> the library's Stage 2 on that list.  Same acceptance rule as the plain forward call."""
+    from paper_2607_27591_b200 import sharded
+    wl, p = toy
+    from tests.gpu_common import dev_bf16
+    k1, k2 = wl.points[50]
+    sh = sharded.ShardedProxFFN(p.D, p.F, dev_bf16(p.bits["wg"]), dev_bf16(p.bits["wu"]), dev_bf16(p.bits["wd"]), 4, 128)
+    try:
+        dg, du, _ = p.quantize(4, 128)
+        for t in (0, 3):
+            sel, y = sh.forward(p.t_x[t], k1, k2)
+            torch.cuda.synchronize()
+            idx, score, sel_ref, thr = p.oracle_stage1(t, k1, k2)
+            sel_np = sel.cpu().numpy().astype(np.int64)
+            check_mask(sel_np, score, sel_ref, thr, k2, p.F)
+            y_ref, _ = po.stage2(p.x[t], sel_np, p.wg, p.wu, p.wd)
+            check_y(y.cpu().numpy(), y_ref)
+    finally:
+        sh.close()
+
+
 def test_calibration_state_matches_the_oracle(pb):
     """Reservoir, quantile and histogram of the library (host side, fed from device buffers) against the oracle's,
     value for value: below and above the capacity, bf16 and fp32 samples, in two pieces."""
