@@ -168,8 +168,17 @@ int ksplit_for(const prox_ffn* h, int B, int n_rows) {
   return ks;
 }
 
+// Function attributes (dynamic shared memory limits) are per device: one flag per (call site, device).
+enum AttrSite { kAtGateupBatch = 0, kAtBatchS1, kAtProxyB4, kAtProxyB8, kAtMma, kAtRows, kAtStage2, kAtFused0, kAtSites = 24 };
+bool& attr_done(int site, int device) {
+  static bool done[kAtSites][64] = {};
+  return done[site][device & 63];
+}
+
 prox_status_t check_common(const prox_ffn* h, const void* x, int B) {
   if (!h || !x) return PROX_ERR_INVALID_ARG;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != h->device) return PROX_ERR_INVALID_ARG;   // the handle's GPU must be current
   if (B < 1 || B > h->cfg.max_batch) return PROX_ERR_INVALID_ARG;
   if (!aligned16(x)) return PROX_ERR_INVALID_ARG;
   return PROX_OK;
@@ -298,7 +307,7 @@ bool batch_path_ok(const prox_ffn* h, int B, bool stage1 = false) {
 prox_status_t launch_union(prox_ffn* h, const int* lists, int stride, const int* cnt, int k, int B, int n,
                            const void* x, int* ulist, int* nu, float* val, cudaStream_t st) {
   const size_t smem = (size_t)(B + 2) * ((n + 31) / 32) * sizeof(unsigned);
-  static bool attr = false;
+  bool& attr = attr_done(kAtStage2, h->device);
   if (!attr) { CK(cudaFuncSetAttribute(union_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
   {
     LaunchScope ls(h, kKUnion, st);
@@ -358,7 +367,7 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     // ranges of (strip, K-block) units per block, then the per-token channel masks
     const size_t lim = (size_t)h->smem_optin - 16384;
     const bool fast_masks = (size_t)D * 2 <= lim && (size_t)F * 4 <= lim;
-    static bool attr_p = false;
+    bool& attr_p = attr_done(kAtBatchS1, h->device);
     if (!attr_p) {
       CK(cudaFuncSetAttribute(proxy_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
       CK(cudaFuncSetAttribute(proxy_umma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
@@ -450,12 +459,12 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
   {
     LaunchScope ls(h, kKProxy, st);
     if (h->bits == 4) {
-      static bool attr4 = false;
+      bool& attr4 = attr_done(kAtProxyB4, h->device);
       if (!attr4) { CK(cudaFuncSetAttribute(proxy_batch_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); attr4 = true; }
       proxy_batch_kernel<4><<<grid, kPBThreads, smem, st>>>(h->P, h->S, h->u_in, h->u_cnt, h->xu, B, D, F, gshift,
                                                            h->part, h->ticket, scores);
     } else {
-      static bool attr8 = false;
+      bool& attr8 = attr_done(kAtProxyB8, h->device);
       if (!attr8) { CK(cudaFuncSetAttribute(proxy_batch_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); attr8 = true; }
       proxy_batch_kernel<8><<<grid, kPBThreads, smem, st>>>(h->P, h->S, h->u_in, h->u_cnt, h->xu, B, D, F, gshift,
                                                            h->part, h->ticket, scores);
@@ -483,7 +492,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   }
   if (mma) {
     // tensor-core path: equal ranges of weight units per block, two blocks per SM for gate/up
-    static bool attr_mma = false;
+    bool& attr_mma = attr_done(kAtMma, h->device);
     if (!attr_mma) {
       CK(cudaFuncSetAttribute(gateup_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
       CK(cudaFuncSetAttribute(down_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
@@ -497,7 +506,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
     {
       LaunchScope ls(h, kKGateUp, st);
       if (D % 512 == 0 && D <= 4096 && ring_slots >= 40) {
-        static bool attr_r = false;
+        bool& attr_r = attr_done(kAtRows, h->device);
         if (!attr_r) {
           CK(cudaFuncSetAttribute(gateup_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
           attr_r = true;
@@ -520,7 +529,7 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
     CK(cudaGetLastError());
   } else {
   const size_t smem = (size_t)B * D * 2;
-  static bool attr = false;
+  bool& attr = attr_done(kAtGateupBatch, h->device);
   if (!attr) { CK(cudaFuncSetAttribute(gateup_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr = true; }
   int blocks = (F + kGBThreads / 32 - 1) / (kGBThreads / 32);
   const int cap = 8 * h->sm_count;
@@ -556,6 +565,7 @@ struct FusedPlan {
   bool ok;
   int grid, pstages, big_bytes, nslots, xch;
   size_t smem;
+  int device;           // the handle's GPU
   int optin;            // the device's opt-in limit: what the kernels' dynamic shared memory attribute is set to
 };
 
@@ -588,14 +598,16 @@ FusedPlan plan_fused(const prox_ffn* h, int k1, int k2, bool thresh = false) {
   pl.xch = D <= 4096 ? 4 : (D <= 8192 ? 2 : 1);          // warp groups of the down projection
   pl.smem = fixed + (size_t)pl.big_bytes;
   pl.optin = h->smem_optin;
+  pl.device = h->device;
   pl.ok = true;
   return pl;
 }
 
 template <int BITS, int NG, bool NORM, bool THRESH>
 cudaError_t launch_fused_tn(const FusedPlan& pl, const FusedParams& prm, cudaStream_t st) {
-  static bool attr_set = false;      // per instantiation; the attribute is per function, not per handle
+  static bool attr_dev[64] = {};     // per instantiation and device: the attribute belongs to the function on a device
   auto kern = prox_fused_kernel<BITS, NG, NORM, THRESH>;
+  bool& attr_set = attr_dev[pl.device & 63];
   if (!attr_set) {
     // the limit, not this plan's size: another handle's shape may need a few bytes more
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.optin);

@@ -36,10 +36,24 @@ def test_noalloc_stage2_matches_handle_based_stage2_twice():
             y_ref = p.y_empty()
             pb.prox_stage2_ffn(p.h, p.t_x[t], 1, sel, k2, y_ref)
             y = torch.full((1, p.D), float("nan"), dtype=torch.float32, device="cuda")
+            y16 = torch.full((1, p.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+            side = torch.cuda.Stream()                 # the second call runs on a stream of its own
+            side.wait_stream(torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            # the driver's own count of free device memory (torch's counter would not see a cudaMalloc inside
+            # the library) and torch's counter (which sees what the binding might allocate)
+            free_before, _ = torch.cuda.mem_get_info()
             before = torch.cuda.memory_allocated()
-            pb.prox_stage2_ffn_noalloc(p.t_x[t], p.t_wg, p.t_wu, w_down_t, p.D, p.F, sel, k2, y, 1)
+            sp = side.cuda_stream if call == 1 else None
+            pb.prox_stage2_ffn_noalloc(p.t_x[t], p.t_wg, p.t_wu, w_down_t, p.D, p.F, sel, k2, y, 1, stream=sp)
+            pb.prox_stage2_ffn_noalloc(p.t_x[t], p.t_wg, p.t_wu, w_down_t, p.D, p.F, sel, k2, y16, 0, stream=sp)
             torch.cuda.synchronize()
             assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.mem_get_info()[0] == free_before, "device memory was allocated during the call"
+            # bf16 output: the fp32 result rounded once
+            a16 = y16.float().cpu().numpy()[0]
+            assert np.all(np.isfinite(a16))
+            assert np.max(np.abs(a16 - y.cpu().numpy()[0])) <= 2.0 ** -8 * np.max(np.abs(y.cpu().numpy()[0])) + 1e-30
             a, b = y.cpu().numpy()[0], y_ref.cpu().numpy()[0]
             assert np.all(np.isfinite(a)), f"call {call}"
             # same kernels, same inputs: only the order of the fp32 atomics may differ
