@@ -53,8 +53,8 @@ struct prox_ffn {
   float* yacc;              // [maxB][D]
   int* dev_status;
   unsigned long long* counters;  // [0] tokens, [1] kept inputs, [2] kept channels
-  unsigned* syncbuf;        // fused kernel: [0..2047] score histogram, [2048] barrier count,
-                            // (64-bit, [2048..2049]), [2050] finish ticket
+  unsigned* syncbuf;        // fused kernel: [0..4095] two score histograms (calls alternate), [4096] barrier count,
+                            // (64-bit, [4096..4097]), [4098] finish ticket
   int smem_optin;           // largest dynamic shared memory a block may ask for
   int coop;                 // device supports cooperative launch
   int sel_unordered;        // the last forward left its mask in the persistent kernel's own order
@@ -674,7 +674,7 @@ prox_status_t launch_fused(prox_ffn* h, const FusedPlan& pl, const void* x, int 
   prm.scores = h->scores; prm.ghist = h->syncbuf; prm.idx_out = h->idx_x;
   prm.spin_limit = h->spin_limit; prm.bar_bias = h->bar_bias; prm.host_flag = h->host_flag_dev;
   prm.sel_out = sel_out; prm.yacc = h->yacc;
-  prm.bar_count = reinterpret_cast<unsigned long long*>(h->syncbuf + 2048); prm.done_ticket = h->syncbuf + 2050;
+  prm.bar_count = reinterpret_cast<unsigned long long*>(h->syncbuf + 4096); prm.done_ticket = h->syncbuf + 4098;
   prm.status = h->dev_status;
   prm.big_bytes = pl.big_bytes; prm.nslots = pl.nslots;
   prm.trace = h->trace;
@@ -724,7 +724,7 @@ prox_status_t forward_kernels(prox_ffn* h, const void* x, int B, int k1, int k2,
 // them back to its idle state (the stream is idle when this runs).
 prox_status_t reset_shared_state(prox_ffn* h, cudaStream_t st) {
   const int ns_max = nstrips_for(h->cfg.d_ff, 8);
-  CK(cudaMemsetAsync(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned), st));
+  CK(cudaMemsetAsync(h->syncbuf, 0, (4096 + 64) * sizeof(unsigned), st));
   CK(cudaMemsetAsync(h->ticket, 0, (size_t)h->cfg.max_batch * ns_max * sizeof(unsigned), st));
   CK(cudaMemsetAsync(h->yacc, 0, (size_t)h->cfg.max_batch * h->cfg.d_model * sizeof(float), st));
   if (h->gacc) {                               // accumulators of the tensor-core batch path (kept at zero between calls)
@@ -792,7 +792,7 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   A(dev_alloc(&h->yacc, (size_t)MB * D));
   A(dev_alloc(&h->dev_status, (size_t)1));
   A(dev_alloc(&h->counters, (size_t)4));
-  A(dev_alloc(&h->syncbuf, (size_t)2048 + 64));
+  A(dev_alloc(&h->syncbuf, (size_t)4096 + 64));
   if (MB > 1) {
     A(dev_alloc(&h->u_in, (size_t)D)); A(dev_alloc(&h->u_ch, (size_t)F)); A(dev_alloc(&h->u_cnt, (size_t)4));
     A(dev_alloc(&h->xu, (size_t)D * kBT)); A(dev_alloc(&h->member, (size_t)F * kBT));
@@ -819,7 +819,7 @@ prox_status_t prox_ffn_create(const prox_ffn_config_t* cfg, const void* w_gate, 
   h->use_fused = 1;
   h->use_union = 1;
   h->use_mma = 1;
-  if (st == PROX_OK) A(cudaMemset(h->syncbuf, 0, (2048 + 64) * sizeof(unsigned)));
+  if (st == PROX_OK) A(cudaMemset(h->syncbuf, 0, (4096 + 64) * sizeof(unsigned)));
   A(dev_alloc(reinterpret_cast<uint16_t**>(&h->x_stage), (size_t)MB * D));
   A(dev_alloc(reinterpret_cast<float**>(&h->y_stage), (size_t)MB * D));
   if (st == PROX_OK) {

@@ -269,6 +269,7 @@ struct FusedSmem {
   int cand2_idx[kCand2Cap];
   int abort_flag;
   int s_last;
+  unsigned call_par;          // parity of the handle's call number: which of the two global histograms is this call's
   unsigned ncand;
   unsigned ncand2;
   unsigned prod_seq;       // rows the producers have armed so far (for the give-up path)
@@ -337,6 +338,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   // global memory is touched before that kernel has completed
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Two global score histograms take turns: this call adds to one and clears the other for the next call (it was
+  // last used by the previous call, which has completed), so nothing is left to clean up when the call ends.
+  // The call number is the barrier counter over the grid size: the counter only grows, by one per block and
+  // call, and this call's own increments cannot complete a multiple of the grid size before every block has
+  // passed this point (each block adds its one after phase B).
+  if (tid == NT - 1) {                          // a thread with no share of the input load below
+    unsigned long long bc;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(bc) : "l"(p.bar_count) : "memory");
+    sm.call_par = (unsigned)((bc / (unsigned long long)G) & 1ull);
+  }
   if (NORM) {
     // FFN input = bf16(RMSNorm(residual stream) * norm weight), the correctly rounded value (the masks
     // depend on it).  Every block does all of it; x and w pass through shared memory once.
@@ -397,6 +408,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  unsigned* const ghist = p.ghist + 2048u * sm.call_par;
+  {
+    unsigned* const other = p.ghist + 2048u * (sm.call_par ^ 1u);
+    const int per = (2048 + G - 1) / G;
+    for (int i = cta * per + tid; i < min(2048, (cta + 1) * per); i += NT) other[i] = 0u;
+  }
   if (warp < 4) {
     // the accumulators of the proxy GEMV start at zero: 16 columns per supergroup, two sets 256 columns apart
     const int ngz = (p.gshift >= 31) ? 1 : (D >> p.gshift);
@@ -739,7 +756,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     if (cta < ntiles) {
       // one atomic per occupied bin and block (thousands of single increments on a few hot bins serialise in L2)
 #pragma unroll 1
-      for (int i = tid; i < 2048; i += NT) { const unsigned v = sm.hist[i]; if (v) atomicAdd(p.ghist + i, v); }
+      for (int i = tid; i < 2048; i += NT) { const unsigned v = sm.hist[i]; if (v) atomicAdd(ghist + i, v); }
     }
     if (warp == 0) tmem_free_all(tbase);
   }
@@ -797,7 +814,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     auto key4_at = [&](int i) -> uint4 {                  // i % 4 == 0
       return in_smem ? lds128(skey_u32 + (uint32_t)i * 4u) : __ldcg(reinterpret_cast<const uint4*>(gkey + i));
     };
-    if (!THRESH && tid < 512) cp_async16(smem_u32(sm.hist) + (uint32_t)tid * 16u, p.ghist + tid * 4);
+    if (!THRESH && tid < 512) cp_async16(smem_u32(sm.hist) + (uint32_t)tid * 16u, ghist + tid * 4);
     cp_async_commit();
     if (in_smem) {
 #pragma unroll 1
@@ -1327,7 +1344,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
           const float4 t = reinterpret_cast<const float4*>(ysum + (size_t)g2 * D)[v4];
           s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
         }
-        atomicAdd(reinterpret_cast<float4*>(p.yacc) + v4, s);
+        // layer form run in place on the residual stream: the block's share of y goes straight into it (every
+        // block read its input before the grid barrier), and there is nothing left to round at the end
+        atomicAdd(reinterpret_cast<float4*>((NORM && p.xres_out == p.xres) ? p.xres_out : p.yacc) + v4, s);
       }
     }
   }
@@ -1355,6 +1374,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
     __syncthreads();
     return;
   }
+  if (NORM && p.xres_out == p.xres) return;     // y went straight into the residual stream: nothing to round, nothing to clean
   if (tid == 0) {
     __threadfence();                            // the block's atomics are out before the ticket is taken
     const unsigned t = atomicAdd(p.done_ticket, 1u);
@@ -1390,7 +1410,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
         }
       }
     }
-    for (int i = tid; i < 2048; i += NT) p.ghist[i] = 0;
     if (tid == 0) *p.done_ticket = 0;
     __syncthreads();
     PROX_TRACE(9);
