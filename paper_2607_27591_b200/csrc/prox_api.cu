@@ -418,14 +418,15 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
         }
         CK(e);
       }
-      direct = fast_masks && !want_scores && h->mask_policy == 0;
+      direct = fast_masks && !want_scores;
       if (!direct) proxy_umma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
     }
     CK(cudaGetLastError());
     if (h->mask_policy == 1) {
       if (!fast_masks) return PROX_ERR_UNSUPPORTED;
       LaunchScope ls(h, kKChannel, st);
-      shared_score_kernel<<<(F + 255) / 256, 256, 0, st>>>(scores, B, F, h->svals);
+      if (direct) shared_score_from_sums_kernel<<<(F + 255) / 256, 256, 0, st>>>(h->pacc, B, F, h->svals);
+      else shared_score_kernel<<<(F + 255) / 256, 256, 0, st>>>(scores, B, F, h->svals);
       batch_channel_mask_kernel<<<1, kFusedThreads, (size_t)F * 4, st>>>(h->svals, F, k2, sel, sel_stride,
                                                                         mark_mask ? h->cmask : nullptr, (1u << B) - 1u, nullptr);
       replicate_mask_kernel<<<(k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B);
@@ -437,7 +438,8 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     {
       LaunchScope ls(h, kKChannel, st);
       batch_channel_mask_kernel<<<B, kFusedThreads, (size_t)F * 4, st>>>(scores, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr, 0u, direct ? h->pacc : nullptr);
+                                                                        mark_mask ? h->cmask : nullptr, 0u,
+                                                                        (direct && h->mask_policy == 0) ? h->pacc : nullptr);
     }
     CK(cudaGetLastError());
     if (mark_mask) h->cmask_marked = 1;

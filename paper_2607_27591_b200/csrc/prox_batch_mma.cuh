@@ -719,4 +719,20 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
   }
 }
 
+// One mask for the whole batch straight from the proxy sums of the tensor-core GEMM: out[j] = sum over the
+// tokens of |up~ SiLU(gate~)|, added token after token in fp32; the accumulator is cleared for the next call.
+__global__ void __launch_bounds__(256) shared_score_from_sums_kernel(float* __restrict__ pacc, int B, int F,
+                                                                     float* __restrict__ out) {
+  const int j = blockIdx.x * 256 + threadIdx.x;
+  if (j >= F) return;
+  float s = 0.f;
+  for (int b = 0; b < kBT; ++b) {
+    float* pg = pacc + (size_t)b * 2 * F + j;
+    const float gate = pg[0], up = pg[F];
+    pg[0] = 0.f; pg[F] = 0.f;
+    if (b < B) s += fabsf(up * silu_fast(gate));
+  }
+  out[j] = s;
+}
+
 }  // namespace prox
