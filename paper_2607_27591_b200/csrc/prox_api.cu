@@ -184,6 +184,27 @@ prox_status_t check_common(const prox_ffn* h, const void* x, int B) {
   return PROX_OK;
 }
 
+// Launch with programmatic stream serialization: the kernel is set up while its predecessor on the stream still
+// runs and waits for it (pdl_enter in the kernel) before it touches anything; the chain of small kernels of the
+// batch path then runs without the launch gaps between them.  Falls back to a plain launch if refused.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  static int use_pdl = getenv("PROX_NO_PDL") ? 0 : 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = use_pdl ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+  if (e != cudaSuccess && use_pdl) {
+    (void)cudaGetLastError();
+    use_pdl = 0; cfg.numAttrs = 0;
+    e = cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+  }
+  return e;
+}
+
 // Brackets one launch with events when the handle's timing hook is on.
 struct LaunchScope {
   prox_ffn* h; cudaStream_t st; ProfRec rec; bool on;
@@ -377,8 +398,8 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     }
     if (fast_masks) {
       LaunchScope ls(h, kKInput, st);
-      batch_input_mask_kernel<<<kBT, kFusedThreads, (size_t)D * 2, st>>>(static_cast<const uint16_t*>(x), B, D, k1,
-                                                                        h->xh, h->tokfac, h->xd, h->soffb);
+      CK(launch_dep(batch_input_mask_kernel, dim3(kBT), dim3(kFusedThreads), (size_t)D * 2, st, static_cast<const uint16_t*>(x), B, D, k1,
+                    h->xh, h->tokfac, h->xd, h->soffb));
     } else {
       if ((s = launch_input_select(h, x, B, k1, 0.f, 0, h->idx_x, D, nullptr, st)) != PROX_OK) return s;
       LaunchScope ls(h, kKInput, st);
@@ -419,17 +440,17 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
         CK(e);
       }
       direct = fast_masks && !want_scores;
-      if (!direct) proxy_umma_finish_kernel<<<2 * h->sm_count, 256, 0, st>>>(h->pacc, B, F, scores);
+      if (!direct) CK(launch_dep(proxy_umma_finish_kernel, dim3(2 * h->sm_count), dim3(256), 0, st, h->pacc, B, F, scores));
     }
     CK(cudaGetLastError());
     if (h->mask_policy == 1) {
       if (!fast_masks) return PROX_ERR_UNSUPPORTED;
       LaunchScope ls(h, kKChannel, st);
-      if (direct) shared_score_from_sums_kernel<<<(F + 255) / 256, 256, 0, st>>>(h->pacc, B, F, h->svals);
-      else shared_score_kernel<<<(F + 255) / 256, 256, 0, st>>>(scores, B, F, h->svals);
-      batch_channel_mask_kernel<<<1, kFusedThreads, (size_t)F * 4, st>>>(h->svals, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr, (1u << B) - 1u, nullptr);
-      replicate_mask_kernel<<<(k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B);
+      if (direct) CK(launch_dep(shared_score_from_sums_kernel, dim3((F + 255) / 256), dim3(256), 0, st, h->pacc, B, F, h->svals));
+      else CK(launch_dep(shared_score_kernel, dim3((F + 255) / 256), dim3(256), 0, st, (const float*)scores, B, F, h->svals));
+      CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kFusedThreads), (size_t)F * 4, st, (const float*)h->svals, F, k2, sel, sel_stride,
+                    mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr));
+      CK(launch_dep(replicate_mask_kernel, dim3((k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B));
       CK(cudaGetLastError());
       if (mark_mask) h->cmask_marked = 1;
       return PROX_OK;
@@ -437,9 +458,8 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     if (!fast_masks) return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
     {
       LaunchScope ls(h, kKChannel, st);
-      batch_channel_mask_kernel<<<B, kFusedThreads, (size_t)F * 4, st>>>(scores, F, k2, sel, sel_stride,
-                                                                        mark_mask ? h->cmask : nullptr, 0u,
-                                                                        (direct && h->mask_policy == 0) ? h->pacc : nullptr);
+      CK(launch_dep(batch_channel_mask_kernel, dim3(B), dim3(kFusedThreads), (size_t)F * 4, st, (const float*)scores, F, k2, sel, sel_stride,
+                    mark_mask ? h->cmask : (unsigned*)nullptr, 0u, (direct && h->mask_policy == 0) ? h->pacc : (float*)nullptr));
     }
     CK(cudaGetLastError());
     if (mark_mask) h->cmask_marked = 1;
@@ -485,9 +505,9 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   if (mma) {
     LaunchScope ls(h, kKUnion, st);
     if (!(marked && h->cmask_marked))
-      union_mark_kernel<<<(B * k2 + 255) / 256, 256, 0, st>>>(sel, sel_stride, k2, B, F, h->cmask, h->dev_status);
+      CK(launch_dep(union_mark_kernel, dim3((B * k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B, F, h->cmask, h->dev_status));
     h->cmask_marked = 0;
-    union_compact_kernel<<<1, 1024, 0, st>>>(h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask);
+    CK(launch_dep(union_compact_kernel, dim3(1), dim3(1024), 0, st, h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask));
     CK(cudaGetLastError());
   } else if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK) {
     return s;
@@ -513,9 +533,10 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
           CK(cudaFuncSetAttribute(gateup_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096));
           attr_r = true;
         }
-        gateup_rows_kernel<<<h->sm_count, kGrThreads, (size_t)ring_slots * row_pitch + (size_t)kMmaWarps * 128 * sizeof(float), st>>>(
-            h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->umask, h->u_cnt + 1, D, ring_slots, h->hb,
-            h->dev_status);
+        CK(launch_dep(gateup_rows_kernel, dim3(h->sm_count), dim3(kGrThreads),
+                      (size_t)ring_slots * row_pitch + (size_t)kMmaWarps * 128 * sizeof(float), st,
+                      h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->umask, h->u_cnt + 1, D, ring_slots, h->hb,
+                      h->dev_status));
       } else {
         gateup_mma_kernel<<<per_sm * h->sm_count, kMmaThreads, mma_smem, st>>>(
             h->wg, h->wu, static_cast<const uint16_t*>(x), B, h->u_ch, h->u_cnt + 1, D, h->gacc);
@@ -525,8 +546,8 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
     CK(cudaGetLastError());
     {
       LaunchScope ls(h, kKDown, st);
-      down_mma_kernel<<<h->sm_count, kMmaThreads, (size_t)kMmaWarps * 512 * sizeof(float), st>>>(
-          h->wdt, h->hb, h->u_ch, h->u_cnt + 1, B, D, h->yacc);
+      CK(launch_dep(down_mma_kernel, dim3(h->sm_count), dim3(kMmaThreads), (size_t)kMmaWarps * 512 * sizeof(float), st,
+                    h->wdt, h->hb, h->u_ch, h->u_cnt + 1, B, D, h->yacc));
     }
     CK(cudaGetLastError());
   } else {
@@ -555,8 +576,8 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   const int n = B * D;
   {
     LaunchScope ls(h, kKFinalize, st);
-    finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(h->yacc, h->fin_resid ? (void*)h->fin_out : y, n,
-                                                     h->cfg.out_dtype, h->fin_resid);
+    CK(launch_dep(finalize_kernel, dim3((n + 255) / 256), dim3(256), 0, st, h->yacc, h->fin_resid ? (void*)h->fin_out : y, n,
+                  h->cfg.out_dtype, (const float*)h->fin_resid));
   }
   CK(cudaGetLastError());
   return PROX_OK;

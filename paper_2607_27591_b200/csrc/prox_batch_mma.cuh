@@ -119,6 +119,7 @@ gateup_mma_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__ 
 __global__ void __launch_bounds__(256)
 union_mark_kernel(const int* __restrict__ lists, int stride, int k, int B, int n, unsigned* __restrict__ mask32,
                   int* __restrict__ status) {
+  pdl_enter();
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= B * k) return;
   const int b = i / k, r = i % k;
@@ -130,6 +131,7 @@ union_mark_kernel(const int* __restrict__ lists, int stride, int k, int B, int n
 __global__ void __launch_bounds__(1024)
 union_compact_kernel(unsigned* __restrict__ mask32, int n, int* __restrict__ ulist, int* __restrict__ nu_out,
                      uint8_t* __restrict__ umask) {
+  pdl_enter();
   __shared__ unsigned long long ws[33];
   const int tid = threadIdx.x;
   const int nw = (n + 3) / 4, per = (nw + 1023) / 1024;          // mask words per thread (consecutive)
@@ -178,6 +180,7 @@ gateup_rows_kernel(const uint16_t* __restrict__ wg, const uint16_t* __restrict__
                    const uint16_t* __restrict__ x, int B, const int* __restrict__ ulist,
                    const uint8_t* __restrict__ umask, const int* __restrict__ nu_ptr, int D, int nslots,
                    float* __restrict__ h_out, int* __restrict__ status) {
+  pdl_enter();
   extern __shared__ __align__(128) uint8_t mm_smem[];
   __shared__ unsigned long long bar_full[kGrMaxSlots / 16], bar_empty[kGrMaxSlots / 16];   // per section of 16 slots
   __shared__ int abort_flag;
@@ -341,6 +344,7 @@ gateup_finish_kernel(float* __restrict__ gacc, const uint8_t* __restrict__ umask
 __global__ void __launch_bounds__(kMmaThreads, 1)
 down_mma_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, const int* __restrict__ ulist,
                 const int* __restrict__ nu_ptr, int B, int D, float* __restrict__ yacc) {
+  pdl_enter();
   extern __shared__ __align__(16) uint8_t mm_smem[];
   float* red = reinterpret_cast<float*>(mm_smem);               // [warps][8 tokens][64 columns]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
@@ -488,7 +492,7 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
   __shared__ int sd[128 * 4];                                     // digit sums of the units of 128 inputs
   constexpr int NT = kFusedThreads;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the proxy GEMM may set up and start on the weights
+  pdl_enter();                                    // the proxy GEMM may set up and start on the weights
   __half* row = xh + (size_t)b * D;
   if (b >= B) {
     if (xd) {
@@ -613,6 +617,7 @@ batch_input_mask_kernel(const uint16_t* __restrict__ x, int B, int D, int k1, __
 // tokens' proxy scores, added token after token in fp32.
 __global__ void __launch_bounds__(256) shared_score_kernel(const float* __restrict__ scores, int B, int F,
                                                            float* __restrict__ out) {
+  pdl_enter();
   const int j = blockIdx.x * 256 + threadIdx.x;
   if (j >= F) return;
   float s = 0.f;
@@ -622,6 +627,7 @@ __global__ void __launch_bounds__(256) shared_score_kernel(const float* __restri
 
 // ... and every token's row of the mask output is that one list.
 __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ sel, int sel_stride, int k2, int B) {
+  pdl_enter();
   const int r = blockIdx.x * 256 + threadIdx.x;
   if (r >= k2) return;
   const int v = sel[r];
@@ -637,6 +643,7 @@ __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ s
 __global__ void __launch_bounds__(kFusedThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
                           unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc) {
+  pdl_enter();
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
   __shared__ unsigned hist[2048], wsum[32], wsum2[32];
@@ -723,6 +730,7 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
 // tokens of |up~ SiLU(gate~)|, added token after token in fp32; the accumulator is cleared for the next call.
 __global__ void __launch_bounds__(256) shared_score_from_sums_kernel(float* __restrict__ pacc, int B, int F,
                                                                      float* __restrict__ out) {
+  pdl_enter();
   const int j = blockIdx.x * 256 + threadIdx.x;
   if (j >= F) return;
   float s = 0.f;

@@ -349,6 +349,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
 // score[b][ch] = |up~ * SiLU(gate~)| from the accumulated sums; the accumulator is cleared for the next call.
 __global__ void __launch_bounds__(256)
 proxy_umma_finish_kernel(float* __restrict__ pacc, int B, int F, float* __restrict__ scores) {
+  pdl_enter();
   for (int i = blockIdx.x * 256 + threadIdx.x; i < kBT * F; i += gridDim.x * 256) {
     const int b = i / F, ch = i - b * F;
     float* pg = pacc + (size_t)b * 2 * F + ch;

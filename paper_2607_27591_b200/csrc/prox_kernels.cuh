@@ -25,6 +25,14 @@ enum DevStatusBits : int { kBadChannel = 1, kBadInput = 2, kWaitExpired = 4 };
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be set up
+// while its predecessor on the stream still runs.  Called first thing: lets the NEXT kernel do the same, then
+// waits until the predecessor has completed and its writes are visible.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ uint4 ld_stream(const void* p) {   // read-once weights: bypass L1
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -741,6 +749,7 @@ down_kernel(const uint16_t* __restrict__ wdt, const float* __restrict__ h, int h
 // With `resid` (layer sub-block form): y = resid + accumulator, fp32 (y may be resid itself).
 __global__ void finalize_kernel(float* __restrict__ yacc, void* y, int n, int out_fp32,
                                 const float* resid = nullptr) {
+  pdl_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const float v = yacc[i];
