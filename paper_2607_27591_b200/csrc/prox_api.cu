@@ -390,8 +390,8 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     const bool fast_masks = (size_t)D * 2 <= lim && (size_t)F * 4 <= lim;
     bool& attr_p = attr_done(kAtBatchS1, h->device);
     if (!attr_p) {
-      CK(cudaFuncSetAttribute(proxy_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
-      CK(cudaFuncSetAttribute(proxy_umma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem));
+      CK(cudaFuncSetAttribute(proxy_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem4));
+      CK(cudaFuncSetAttribute(proxy_umma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBuSmem8));
       CK(cudaFuncSetAttribute(batch_input_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
       CK(cudaFuncSetAttribute(batch_channel_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
       attr_p = true;
@@ -415,7 +415,7 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
       if (usplit < 1) usplit = 1;
       const int nitems = ntiles * usplit;
       const int grid = nitems < h->sm_count ? nitems : h->sm_count;
-      const size_t smem = (size_t)kBuSmem;
+      const size_t smem = (size_t)(h->bits == 4 ? kBuSmem4 : kBuSmem8);
       if ((s = ensure_pmap(h, row_bytes)) != PROX_OK) return s;
       {
         // programmatic dependent launch: the kernel sets up and requests its first weight tiles while the

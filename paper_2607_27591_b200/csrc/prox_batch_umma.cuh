@@ -13,10 +13,10 @@
 // nothing else touches the bytes: a worker warp waits for the stage and issues the MMA.  For 4-bit
 // codes the worker first writes the tile with the high nibbles masked off into a second buffer (the
 // operand of the second MMA).  B operand of a block: row k = 8 tokens x 4 digits = 32 bytes (N = 32).
-// A unit = 128 consecutive inputs (4 blocks): its MMAs accumulate into one of two 64-column sets of
-// tensor memory (32 columns for the bytes, 32 for the low nibbles; a unit's first MMA overwrites them); eight read-back warps
-// per set apply the unit's scales while the workers already fill the other set.  Items = (128-byte tile of the rows, range of
-// units); an item's partial sums are added to an fp32 accumulator in global memory, a small kernel forms
+// A unit = 128 consecutive inputs (4 blocks): its MMAs accumulate into one of four 64-column sets of
+// tensor memory (32 columns for the bytes, 32 for the low nibbles; a unit's first MMA overwrites them); two groups
+// of eight read-back warps take turns on the units and apply their scales while the workers already fill
+// the other sets.  Items = (128-byte tile of the rows, range of units); an item's partial sums are added to an fp32 accumulator in global memory, a small kernel forms
 // the scores.
 #pragma once
 
@@ -29,9 +29,11 @@ namespace prox {
 constexpr int kBuWorkers = 8;                        // warps 1..8: (mask the low nibbles,) issue the MMAs
 constexpr int kBuRb = 16;                            // warps 9..24: read the accumulators back (eight per accumulator set)
 constexpr int kBuThreads = (1 + kBuWorkers + kBuRb) * 32;
-constexpr int kBuStages = 6;                         // stage = one unit (four blocks); even: a stage always meets the same workers
+constexpr int kBuStages4 = 8, kBuStages8 = 10;       // stage = one unit (four blocks); even: a stage always meets the same workers
+constexpr int kBuStagesMax = 10;                     // (8-bit codes need no low-nibble buffers: two stages more)
 constexpr int kBuTile = 4096, kBuDig = 1024;         // block: 32 rows x 128 bytes | 32 rows x 32 digit bytes
-constexpr int kBuSmem = 1024 + kBuStages * 4 * (kBuTile + kBuDig) + kBuWorkers * kBuTile;
+constexpr int kBuSmem4 = 1024 + kBuStages4 * 4 * (kBuTile + kBuDig) + kBuWorkers * kBuTile;
+constexpr int kBuSmem8 = 1024 + kBuStages8 * 4 * (kBuTile + kBuDig);
 
 __device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
@@ -96,8 +98,9 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
                   float* __restrict__ pacc, int* __restrict__ status) {
   constexpr bool LO = BITS == 4;
   constexpr int CH = LO ? 16 : 8;
+  constexpr int kBuStages = LO ? kBuStages4 : kBuStages8;
   extern __shared__ __align__(128) uint8_t bu_smem[];
-  __shared__ unsigned long long full[kBuStages], empty[kBuStages], gdone[2];
+  __shared__ unsigned long long full[kBuStagesMax], empty[kBuStagesMax], gdone[4];
   __shared__ unsigned drained[kBuRb];                 // per read-back warp: units it has read back and cleared
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
@@ -107,15 +110,15 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
   const int nunits = D >> 7;                          // units of 128 inputs
   const uint32_t raw0 = (smem_u32(bu_smem) + 1023u) & ~1023u;           // [stages][4][4096] tiles as TMA writes them
   const uint32_t lo0 = raw0 + (uint32_t)(kBuStages * 4 * kBuTile);      // [workers][4096] low-nibble copies
-  const uint32_t dig0 = lo0 + (uint32_t)(kBuWorkers * kBuTile);         // [stages][4][1024] digit rows
+  const uint32_t dig0 = lo0 + (uint32_t)(LO ? kBuWorkers * kBuTile : 0);         // [stages][4][1024] digit rows
   volatile int* abortp = &abort_flag;
   if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&pmap) : "memory");
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(128u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid < kBuStages) { mbar_init(smem_u32(&full[tid]), 1); mbar_init(smem_u32(&empty[tid]), 1); }
-  if (tid < 2) mbar_init(smem_u32(&gdone[tid]), 1);
+  if (tid < 4) mbar_init(smem_u32(&gdone[tid]), 1);
   if (tid < kBuRb) drained[tid] = 0u;
   if (tid == 0) abort_flag = 0;
   fence_mbar_init();
@@ -126,7 +129,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
   const int rb = warp - 1 - kBuWorkers;               // read-back warp: set rb / 8, tokens 4 * (rb / 4 % 2) .., lanes 32 * (warp % 4) ..
   const int nitems = ntiles * usplit;
   if (tid != 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // thread 0 (the producer) first requests weights
-  unsigned gseq = 0;                                  // units this CTA has started (for the two accumulator sets)
+  unsigned gseq = 0;                                  // units this CTA has started (unit number modulo 4 = accumulator set)
   if (warp == 0) {
     // ---- producer: one lane keeps the ring full
     if (lane == 0) {
@@ -176,12 +179,12 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
       }
     }
   } else if (rb < 0) {
-    // ---- workers: group w / 4 owns the units with number gs % 2 == w / 4 (accumulator set w / 4).  4-bit codes:
+    // ---- workers: group w / 4 owns the units with number gs % 2 == w / 4 (accumulator sets gs % 4).  4-bit codes:
     // each warp of the group writes the low nibbles of one block of the unit, then the group's first warp
     // issues the unit's MMAs, the first of them overwriting the accumulators.  8-bit codes: only that warp works.
-    const int w = warp - 1, wj = w & 3, set = w >> 2;
+    const int w = warp - 1, wj = w & 3, grp = w >> 2;
     const uint32_t lob = lo0 + (uint32_t)w * (uint32_t)kBuTile;
-    const uint32_t lo_group = lo0 + (uint32_t)(set * 4) * (uint32_t)kBuTile;
+    const uint32_t lo_group = lo0 + (uint32_t)(grp * 4) * (uint32_t)kBuTile;
     constexpr uint32_t idesc = umma_idesc_u8s8(128, 32);
     unsigned mine = 0, s_prev = 0, use_prev = 0;
     bool bad = false;                                 // a wait of this warp gave up; the group leaves together
@@ -192,8 +195,9 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
         const int u0 = (int)(((long long)nunits * part) / usplit), u1 = (int)(((long long)nunits * (part + 1)) / usplit);
         bool dead = false;
 #pragma unroll 1
-        for (int ul = (int)(((unsigned)set + gseq) & 1u); ul < u1 - u0; ul += 2) {
+        for (int ul = (int)(((unsigned)grp + gseq) & 1u); ul < u1 - u0; ul += 2) {
           const unsigned gs = gseq + (unsigned)ul, s = gs % kBuStages, use = gs / kBuStages;
+          const int set = (int)(gs & 3u);              // four accumulator sets: a group alternates between two of them
           const uint32_t raws = raw0 + s * (uint32_t)(4 * kBuTile);
           bad = bad || !__all_sync(0xffffffffu, mbar_wait(smem_u32(&full[s]), use & 1u, abortp));
           if (LO) {
@@ -212,7 +216,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
             }
             uint32_t any_bad;                         // barrier of the group's 128 threads that also ORs the flags
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(any_bad) : "r"((uint32_t)bad), "r"(2 + set) : "memory");
+                         : "=r"(any_bad) : "r"((uint32_t)bad), "r"(2 + grp) : "memory");
             if (any_bad) { dead = true; break; }
           } else if (bad) { dead = true; break; }
           ++mine; s_prev = s; use_prev = use;
@@ -220,13 +224,13 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
           // the set must have been read back by its read-back warps: counters, not an mbarrier phase; lanes 0..7
           // each watch one read-back warp of the set
           bool set_ok = true;
-          if (gs >= 2u) {
+          if (gs >= 4u) {
             set_ok = false;
 #pragma unroll 1
             for (unsigned it = 0; it < kSpinLimit; ++it) {
               unsigned seen = gs;
-              if (lane < 8) asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(seen) : "r"(smem_u32(&drained[set * 8 + lane])) : "memory");
-              if (__all_sync(0xffffffffu, (int)(seen - (gs - 1u)) >= 0)) { set_ok = true; break; }
+              if (lane < 8) asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(seen) : "r"(smem_u32(&drained[grp * 8 + lane])) : "memory");
+              if (__all_sync(0xffffffffu, (int)(seen - (gs - 3u)) >= 0)) { set_ok = true; break; }   // unit gs - 4 read back
               __nanosleep(20);
               if ((it & 255u) == 255u && *abortp) break;
             }
@@ -264,7 +268,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
     }
   } else {
     // ---- read-back: thread = byte column of the tile and four of the tokens; per unit 4 x (bytes, low nibbles) x 4 digits
-    const int q4 = warp & 3, half = (rb >> 2) & 1, set = rb >> 3, col = q4 * 32 + lane;
+    const int q4 = warp & 3, half = (rb >> 2) & 1, grp = rb >> 3, col = q4 * 32 + lane;
     float tf[4];
 #pragma unroll
     for (int b = 0; b < 4; ++b) tf[b] = tokfac[half * 4 + b] * 9.094947017729282e-13f;   // * 2^-40
@@ -288,7 +292,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
         if (ul >= nu) return make_float4(0.f, 0.f, 0.f, 0.f);
         return __ldg(reinterpret_cast<const float4*>(soff + (size_t)(u0 + ul) * kBT) + half);
       };
-      const int ul0 = (int)(((unsigned)set + gseq) & 1u);            // this set's first unit of the item
+      const int ul0 = (int)(((unsigned)grp + gseq) & 1u);            // this group's first unit of the item
       uint32_t scw = load_scale(ul0);
       float4 so4 = load_so(ul0);
 #pragma unroll 1
@@ -297,7 +301,8 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
         const uint32_t scw2 = load_scale(ul + 2);
         const float4 so42 = load_so(ul + 2);
         const float so[4] = {so4.x, so4.y, so4.z, so4.w};
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&gdone[set]), (gs >> 1) & 1u, abortp))) { dead = true; break; }
+        const int set = (int)(gs & 3u);
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&gdone[set]), (gs >> 2) & 1u, abortp))) { dead = true; break; }
         tc_fence_after();
         const uint32_t ta = tbase + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(set * 64 + half * 16);
         uint32_t a[16], l[16];
@@ -343,7 +348,7 @@ proxy_umma_kernel(const __grid_constant__ CUtensorMap pmap, const __half* __rest
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && abort_flag) atomicOr(status, kWaitExpired);
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(128u) : "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(256u) : "memory");
 }
 
 // score[b][ch] = |up~ * SiLU(gate~)| from the accumulated sums; the accumulator is cleared for the next call.
