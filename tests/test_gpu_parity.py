@@ -465,6 +465,8 @@ def test_fused_all_zero_input(pb, toy):
     (128, 40960, 38, 39000, 4, 128),       # scores in shared memory, more than 256 channels per block
     (8192, 320, 2458, 75, 8, 128),         # ragged last strip, 8-bit codes, two down-projection groups
     (384, 448, 115, 104, 4, 128),          # sizes that are no multiple of the strip or chunk steps
+    (128, 64, 38, 15, 4, 0),               # the smallest layer the library takes (a proxy row is half a tile wide)
+    (256, 64, 77, 15, 8, 128),             # ... with 8-bit codes and two scale groups
 ])
 def test_extreme_shapes(pb, D, F, k1, k2, bits, group):
     wg, wu, wd, x = inputs.make_small(D, F, 3, seed=D + F)
