@@ -507,7 +507,13 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
     if (!(marked && h->cmask_marked))
       CK(launch_dep(union_mark_kernel, dim3((B * k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B, F, h->cmask, h->dev_status));
     h->cmask_marked = 0;
-    CK(launch_dep(union_compact_kernel, dim3(1), dim3(1024), 0, st, h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask));
+    {
+      const size_t need = (size_t)F * 5 + 16;
+      const int staged = need <= (size_t)h->smem_optin - 4096 ? 1 : 0;
+      bool& attr_u = attr_done(kAtFused0, h->device);
+      if (!attr_u) { CK(cudaFuncSetAttribute(union_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 4096)); attr_u = true; }
+      CK(launch_dep(union_compact_kernel, dim3(1), dim3(1024), staged ? need : (size_t)0, st, h->cmask, F, h->u_ch, h->u_cnt + 1, h->umask, staged));
+    }
     CK(cudaGetLastError());
   } else if ((s = launch_union(h, sel, sel_stride, nullptr, k2, B, F, nullptr, h->u_ch, h->u_cnt + 1, h->member, st)) != PROX_OK) {
     return s;

@@ -130,29 +130,46 @@ union_mark_kernel(const int* __restrict__ lists, int stride, int k, int B, int n
 
 __global__ void __launch_bounds__(1024)
 union_compact_kernel(unsigned* __restrict__ mask32, int n, int* __restrict__ ulist, int* __restrict__ nu_out,
-                     uint8_t* __restrict__ umask) {
+                     uint8_t* __restrict__ umask, int staged) {
   pdl_enter();
+  // staged: the list is put together in shared memory (a thread's entries land anywhere in it) and leaves in
+  // whole lines; otherwise (a layer too wide for that) the entries go to global memory one by one
+  extern __shared__ __align__(16) uint8_t uc_smem[];
+  int* slist = staged ? reinterpret_cast<int*>(uc_smem) : ulist;              // [n] channel ids
+  uint8_t* smask = staged ? uc_smem + (size_t)n * 4 : umask;                  // [n] token bits
   __shared__ unsigned long long ws[33];
   const int tid = threadIdx.x;
-  const int nw = (n + 3) / 4, per = (nw + 1023) / 1024;          // mask words per thread (consecutive)
+  const int nw = (n + 3) / 4, per = (nw + 1023) / 1024;          // mask words per thread (consecutive), at most 16
   const int w0 = min(nw, tid * per), w1 = min(nw, w0 + per);
+  unsigned m[16];
   unsigned cnt = 0;
-  for (int w = w0; w < w1; ++w) {
-    const unsigned m = mask32[w];
-    cnt += ((m & 0xffu) ? 1u : 0u) + ((m & 0xff00u) ? 1u : 0u) + ((m & 0xff0000u) ? 1u : 0u) + ((m >> 24) ? 1u : 0u);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    m[i] = (w0 + i < w1) ? __ldcg(mask32 + w0 + i) : 0u;
+    cnt += ((m[i] & 0xffu) ? 1u : 0u) + ((m[i] & 0xff00u) ? 1u : 0u) + ((m[i] & 0xff0000u) ? 1u : 0u) + ((m[i] >> 24) ? 1u : 0u);
   }
   unsigned long long tot;
   unsigned pos = (unsigned)block_scan_excl<1024>((unsigned long long)cnt, ws, &tot);
-  for (int w = w0; w < w1; ++w) {
-    const unsigned m = mask32[w];
-    mask32[w] = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const unsigned by = (m >> (8 * q)) & 0xffu;
-      if (by && w * 4 + q < n) { ulist[pos] = w * 4 + q; umask[pos] = (uint8_t)by; ++pos; }
+  for (int i = 0; i < 16; ++i) {
+    if (w0 + i < w1) {
+      mask32[w0 + i] = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const unsigned by = (m[i] >> (8 * q)) & 0xffu;
+        const int ch = (w0 + i) * 4 + q;
+        if (by && ch < n) { slist[pos] = ch; smask[pos] = (uint8_t)by; ++pos; }
+      }
     }
   }
-  if (tid == 0) *nu_out = (int)tot;
+  __syncthreads();
+  const int nu = (int)tot;
+  if (staged) {
+    for (int i = tid; i < nu; i += 1024) ulist[i] = slist[i];
+    for (int i = tid; i < (nu + 3) / 4; i += 1024)               // four bytes at a time (the tail may carry stale bytes: unused)
+      reinterpret_cast<unsigned*>(umask)[i] = reinterpret_cast<const unsigned*>(smask)[i];
+  }
+  if (tid == 0) *nu_out = nu;
 }
 
 // ----------------------------------------------------------------------------
