@@ -659,7 +659,7 @@ __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ s
 // over the summed scores) the kept channels get all of token_bits.
 __global__ void __launch_bounds__(kFusedThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
-                          unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc) {
+                          unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc, int nrep) {
   pdl_enter();
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
@@ -735,11 +735,19 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
       const bool gt = k4[e] > T, eq = k4[e] == T;
       if (gt || (eq && re < quota)) {
         const int ch = q * 4 + e;
-        out[rg + min(re, quota)] = ch;
+        if (nrep > 1) reinterpret_cast<int*>(skey + F)[rg + min(re, quota)] = ch;     // staged: every token's row gets the list
+        else out[rg + min(re, quota)] = ch;
         if (cmask) atomicOr(cmask + (ch >> 2), (token_bits ? token_bits : (1u << b)) << (8 * (ch & 3)));
       }
       rg += gt ? 1u : 0u; re += eq ? 1u : 0u;
     }
+  }
+  if (nrep > 1) {
+    // one mask for the batch: the list goes to every token's row, in whole lines
+    __syncthreads();
+    const int* slist = reinterpret_cast<const int*>(skey + F);
+    for (int r = 0; r < nrep; ++r)
+      for (int i = tid; i < k2; i += NT) sel_out[(size_t)r * sel_stride + i] = slist[i];
   }
 }
 
