@@ -443,6 +443,50 @@ def test_batch_random_budgets(pb, toy):
     assert pb.prox_last_device_status(p.h) == 0
 
 
+@pytest.mark.parametrize("bits,group", [(4, 0), (4, 128), (8, 0), (8, 128)])
+def test_batch_edge_budgets_and_scores_all_formats(pb, toy, bits, group):
+    """The tensor-core Stage 1 of the batch path at the corners of the budget, for every integer format: masks and
+    outputs through the forward call, and the scores themselves (asked for explicitly) against the oracle."""
+    wl, p = toy
+    dg, du, _ = p.quantize(bits, group)
+    for B, t0 in ((2, 0), (8, 5)):
+        for k1, k2 in ((p.D, p.F), (1, 1), (p.D, 1), (17, p.F - 1), (154, 358)):
+            _forward_check(pb, p, t0, k1, k2, B=B)
+        k1, k2 = 154, 358
+        sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        sc = torch.empty(B, p.F, dtype=torch.float32, device="cuda")
+        pb.prox_stage1_mask(p.h, p.t_x[t0:t0 + B], B, k1, k2, sel, sc)
+        torch.cuda.synchronize()
+        for b in range(B):
+            idx, score, sel_ref, thr = p.oracle_stage1(t0 + b, k1, k2)
+            assert float(np.max(np.abs(sc.cpu().numpy()[b] - score)) / thr) < 2e-4
+    assert pb.prox_last_device_status(p.h) == 0
+
+
+@pytest.mark.parametrize("bits,group,B", [(4, 128, 5), (8, 0, 8), (4, 0, 2)])
+def test_batch_stage1_over_several_units_and_items(pb, bits, group, B):
+    """A layer wide and deep enough that a block of the batched proxy GEMM takes several items of several units
+    each (reuse of ring stages and of the accumulator sets): scores and masks against the oracle."""
+    D, F, k1, k2 = 2048, 4096, 614, 942
+    wg, wu, wd, x = inputs.make_small(D, F, 9, seed=D + F + bits)
+    p = Problem(pb, wg, wu, wd, x, max_batch=8)
+    try:
+        p.quantize(bits, group)
+        sel = torch.empty(B, k2, dtype=torch.int32, device="cuda")
+        sc = torch.empty(B, F, dtype=torch.float32, device="cuda")
+        for rep in range(2):                        # twice: the accumulator in global memory must come back clean
+            pb.prox_stage1_mask(p.h, p.t_x[:B], B, k1, k2, sel, sc)
+            torch.cuda.synchronize()
+            for b in range(B):
+                idx, score, sel_ref, thr = p.oracle_stage1(b, k1, k2)
+                assert float(np.max(np.abs(sc.cpu().numpy()[b] - score)) / thr) < 2e-4, (rep, b)
+                check_mask(sel.cpu().numpy()[b].astype(np.int64), score, sel_ref, thr, k2, F)
+        _forward_check(pb, p, 1, k1, k2, B=B)
+        assert pb.prox_last_device_status(p.h) == 0
+    finally:
+        p.close()
+
+
 def test_fused_all_zero_input(pb, toy):
     """x = 0: every score ties at 0; the mask must be the first k2 channels and y = 0."""
     wl, p = toy
