@@ -668,26 +668,45 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned* gkey = reinterpret_cast<const unsigned*>(scores) + (size_t)b * F;
   const uint32_t skey_u32 = smem_u32(skey);
+  for (int i = tid; i < 2048; i += NT) hist[i] = 0;
+  __syncthreads();
   if (pacc) {
-    // scores straight from the proxy sums of the tensor-core GEMM ([token][gate | up][channel]); the
-    // token's entries are cleared for the next call
+    // scores straight from the proxy sums of the tensor-core GEMM ([token][gate | up][channel]); the token's
+    // entries are cleared for the next call.  Four rounds of loads are issued before the first use: one round per
+    // dependent iteration would put the latency of global memory on every one of them.
     float4* pg = reinterpret_cast<float4*>(pacc + (size_t)b * 2 * F);
     float4* pu = pg + F / 4;
-    for (int i = tid; i < F / 4; i += NT) {
-      const float4 g = pg[i], u = pu[i];
-      pg[i] = make_float4(0.f, 0.f, 0.f, 0.f); pu[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      reinterpret_cast<uint4*>(skey)[i] = make_uint4(__float_as_uint(fabsf(u.x * silu_fast(g.x))), __float_as_uint(fabsf(u.y * silu_fast(g.y))),
-                                                     __float_as_uint(fabsf(u.z * silu_fast(g.z))), __float_as_uint(fabsf(u.w * silu_fast(g.w))));
+    const int n4 = F / 4;
+#pragma unroll 1
+    for (int i0 = tid; i0 < n4; i0 += 4 * NT) {
+      float4 g[4], u[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = i0 + r * NT;
+        g[r] = i < n4 ? __ldcg(pg + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        u[r] = i < n4 ? __ldcg(pu + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = i0 + r * NT;
+        if (i < n4) {
+          pg[i] = make_float4(0.f, 0.f, 0.f, 0.f); pu[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          const uint4 k = make_uint4(__float_as_uint(fabsf(u[r].x * silu_fast(g[r].x))), __float_as_uint(fabsf(u[r].y * silu_fast(g[r].y))),
+                                     __float_as_uint(fabsf(u[r].z * silu_fast(g[r].z))), __float_as_uint(fabsf(u[r].w * silu_fast(g[r].w))));
+          reinterpret_cast<uint4*>(skey)[i] = k;
+          atomicAdd(&hist[k.x >> 20], 1u); atomicAdd(&hist[k.y >> 20], 1u);
+          atomicAdd(&hist[k.z >> 20], 1u); atomicAdd(&hist[k.w >> 20], 1u);
+        }
+      }
     }
   } else {
     for (int i = tid; i < F / 4; i += NT) cp_async16(skey_u32 + (uint32_t)i * 16u, gkey + 4 * i);
     cp_async_commit();
-  }
-  for (int i = tid; i < 2048; i += NT) hist[i] = 0;
-  cp_async_wait<0>();
-  __syncthreads();
+    cp_async_wait<0>();
+    __syncthreads();
 #pragma unroll 1
-  for (int i = tid; i < F; i += NT) atomicAdd(&hist[skey[i] >> 20], 1u);
+    for (int i = tid; i < F; i += NT) atomicAdd(&hist[skey[i] >> 20], 1u);
+  }
   __syncthreads();
   unsigned ab;
   unsigned prefix = kth_in_block<4, false>(hist, (unsigned)k2, wsum, lane, warp, &ab);
@@ -758,12 +777,19 @@ __global__ void __launch_bounds__(256) shared_score_from_sums_kernel(float* __re
   pdl_enter();
   const int j = blockIdx.x * 256 + threadIdx.x;
   if (j >= F) return;
+  // all loads first (a load behind every store would put the latency of global memory on every token)
+  float gate[kBT], up[kBT];
+#pragma unroll
+  for (int b = 0; b < kBT; ++b) {
+    const float* pg = pacc + (size_t)b * 2 * F + j;
+    gate[b] = __ldcg(pg); up[b] = __ldcg(pg + F);
+  }
   float s = 0.f;
+#pragma unroll
   for (int b = 0; b < kBT; ++b) {
     float* pg = pacc + (size_t)b * 2 * F + j;
-    const float gate = pg[0], up = pg[F];
     pg[0] = 0.f; pg[F] = 0.f;
-    if (b < B) s += fabsf(up * silu_fast(gate));
+    if (b < B) s += fabsf(up[b] * silu_fast(gate[b]));
   }
   out[j] = s;
 }
