@@ -450,10 +450,10 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
       else CK(launch_dep(shared_score_kernel, dim3((F + 255) / 256), dim3(256), 0, st, (const float*)scores, B, F, h->svals));
       if ((size_t)F * 4 + (size_t)k2 * 4 <= lim) {
         // the one block also writes the list into every token's row
-        CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kFusedThreads), (size_t)F * 4 + (size_t)k2 * 4, st, (const float*)h->svals, F, k2, sel,
+        CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kCmThreads), (size_t)F * 4 + (size_t)k2 * 4, st, (const float*)h->svals, F, k2, sel,
                       sel_stride, mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, B));
       } else {
-        CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kFusedThreads), (size_t)F * 4, st, (const float*)h->svals, F, k2, sel, sel_stride,
+        CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kCmThreads), (size_t)F * 4, st, (const float*)h->svals, F, k2, sel, sel_stride,
                       mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, 1));
         CK(launch_dep(replicate_mask_kernel, dim3((k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B));
       }
@@ -464,7 +464,7 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     if (!fast_masks) return launch_channel_select(h, scores, B, k2, 0.f, 0, sel, sel_stride, nullptr, st);
     {
       LaunchScope ls(h, kKChannel, st);
-      CK(launch_dep(batch_channel_mask_kernel, dim3(B), dim3(kFusedThreads), (size_t)F * 4, st, (const float*)scores, F, k2, sel, sel_stride,
+      CK(launch_dep(batch_channel_mask_kernel, dim3(B), dim3(kCmThreads), (size_t)F * 4, st, (const float*)scores, F, k2, sel, sel_stride,
                     mark_mask ? h->cmask : (unsigned*)nullptr, 0u, (direct && h->mask_policy == 0) ? h->pacc : (float*)nullptr, 1));
     }
     CK(cudaGetLastError());

@@ -657,14 +657,15 @@ __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ s
 // byte of cmask (the union of the tokens' masks is read off those bytes).
 // token_bits = 0: block b is token b and sets bit b.  Otherwise (one shared mask for the batch: one block
 // over the summed scores) the kept channels get all of token_bits.
-__global__ void __launch_bounds__(kFusedThreads)
+constexpr int kCmThreads = 1024;                   // channel-mask kernel: all 32 warps of a block
+__global__ void __launch_bounds__(kCmThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
                           unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc, int nrep) {
   pdl_enter();
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
   __shared__ unsigned hist[2048], wsum[32], wsum2[32];
-  constexpr int NT = kFusedThreads;
+  constexpr int NT = kCmThreads;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned* gkey = reinterpret_cast<const unsigned*>(scores) + (size_t)b * F;
   const uint32_t skey_u32 = smem_u32(skey);
