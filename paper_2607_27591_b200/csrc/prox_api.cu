@@ -451,10 +451,15 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
       if ((size_t)F * 4 + (size_t)k2 * 4 <= lim) {
         // the one block also writes the list into every token's row
         CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kCmThreads), (size_t)F * 4 + (size_t)k2 * 4, st, (const float*)h->svals, F, k2, sel,
-                      sel_stride, mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, B));
+                      sel_stride, (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, B, mark_mask ? h->u_ch : (int*)nullptr, h->umask,
+                      h->u_cnt + 1));
+        CK(cudaGetLastError());
+        if (mark_mask) h->cmask_marked = 2;          // the union is listed already: it is the mask itself
+        return PROX_OK;
       } else {
         CK(launch_dep(batch_channel_mask_kernel, dim3(1), dim3(kCmThreads), (size_t)F * 4, st, (const float*)h->svals, F, k2, sel, sel_stride,
-                      mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, 1));
+                      mark_mask ? h->cmask : (unsigned*)nullptr, (1u << B) - 1u, (float*)nullptr, 1, (int*)nullptr, (uint8_t*)nullptr,
+                      (int*)nullptr));
         CK(launch_dep(replicate_mask_kernel, dim3((k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B));
       }
       CK(cudaGetLastError());
@@ -465,7 +470,8 @@ prox_status_t launch_stage1_batch(prox_ffn* h, const void* x, int B, int k1, int
     {
       LaunchScope ls(h, kKChannel, st);
       CK(launch_dep(batch_channel_mask_kernel, dim3(B), dim3(kCmThreads), (size_t)F * 4, st, (const float*)scores, F, k2, sel, sel_stride,
-                    mark_mask ? h->cmask : (unsigned*)nullptr, 0u, (direct && h->mask_policy == 0) ? h->pacc : (float*)nullptr, 1));
+                    mark_mask ? h->cmask : (unsigned*)nullptr, 0u, (direct && h->mask_policy == 0) ? h->pacc : (float*)nullptr, 1,
+                    (int*)nullptr, (uint8_t*)nullptr, (int*)nullptr));
     }
     CK(cudaGetLastError());
     if (mark_mask) h->cmask_marked = 1;
@@ -510,10 +516,11 @@ prox_status_t launch_stage2_batch(prox_ffn* h, const void* x, int B, const int* 
   const bool mma = stage2_mma_ok(h);
   if (mma) {
     LaunchScope ls(h, kKUnion, st);
-    if (!(marked && h->cmask_marked))
-      CK(launch_dep(union_mark_kernel, dim3((B * k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B, F, h->cmask, h->dev_status));
+    const int listed = marked ? h->cmask_marked : 0;       // 1: bits set by Stage 1 of this call, 2: the union list is there already
     h->cmask_marked = 0;
-    {
+    if (!listed)
+      CK(launch_dep(union_mark_kernel, dim3((B * k2 + 255) / 256), dim3(256), 0, st, sel, sel_stride, k2, B, F, h->cmask, h->dev_status));
+    if (listed != 2) {
       const size_t need = (size_t)F * 5 + 16;
       const int staged = need <= (size_t)h->smem_optin - 4096 ? 1 : 0;
       bool& attr_u = attr_done(kAtFused0, h->device);

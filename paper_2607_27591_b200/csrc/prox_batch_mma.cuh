@@ -660,7 +660,8 @@ __global__ void __launch_bounds__(256) replicate_mask_kernel(int* __restrict__ s
 constexpr int kCmThreads = 1024;                   // channel-mask kernel: all 32 warps of a block
 __global__ void __launch_bounds__(kCmThreads)
 batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* __restrict__ sel_out, int sel_stride,
-                          unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc, int nrep) {
+                          unsigned* __restrict__ cmask, unsigned token_bits, float* __restrict__ pacc, int nrep,
+                          int* __restrict__ ulist, uint8_t* __restrict__ umask, int* __restrict__ nu_out) {
   pdl_enter();
   extern __shared__ __align__(16) uint8_t bm_smem[];
   unsigned* skey = reinterpret_cast<unsigned*>(bm_smem);         // [F] score bits
@@ -768,6 +769,11 @@ batch_channel_mask_kernel(const float* __restrict__ scores, int F, int k2, int* 
     const int* slist = reinterpret_cast<const int*>(skey + F);
     for (int r = 0; r < nrep; ++r)
       for (int i = tid; i < k2; i += NT) sel_out[(size_t)r * sel_stride + i] = slist[i];
+    if (ulist) {
+      // ... and it is the union of the tokens' masks as well: every kept channel belongs to every token
+      for (int i = tid; i < k2; i += NT) { ulist[i] = slist[i]; umask[i] = (uint8_t)token_bits; }
+      if (tid == 0) *nu_out = k2;
+    }
   }
 }
 
