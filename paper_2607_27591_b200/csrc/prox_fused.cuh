@@ -768,8 +768,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   fence_proxy_async();                        // phase B's plain accesses to the big buffer come before the ring's bulk copies
   __syncthreads();
   if (tid == 0) {
-    __threadfence();                          // cumulative: publishes the block's writes seen through the barrier above
-    const unsigned long long old = atomicAdd(p.bar_count, 1ull);
+    // release (cumulative): publishes the block's writes seen through the barrier above
+    unsigned long long old;
+    asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.bar_count) : "memory");
     // the count is reset by the host long before 2^32 calls; the low word is enough for the division
     const unsigned long long target = old - (unsigned long long)((unsigned)old % (unsigned)G) + (unsigned long long)G +
                                       (unsigned long long)p.bar_bias;
@@ -782,7 +783,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
       if (!ok && it > 64) __nanosleep(32);
     }
     if (!ok) { sm.abort_flag = 1; atomicOr(p.status, kWaitExpired); if (p.host_flag) *reinterpret_cast<volatile int*>(p.host_flag) = 1; }
-    __threadfence();
   }
   __syncthreads();
   const bool alive = sm.abort_flag == 0;      // block-uniform; a dead block skips to the end
@@ -1376,10 +1376,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) prox_fused_kernel(const Fuse
   }
   if (NORM && p.xres_out == p.xres) return;     // y went straight into the residual stream: nothing to round, nothing to clean
   if (tid == 0) {
-    __threadfence();                            // the block's atomics are out before the ticket is taken
-    const unsigned t = atomicAdd(p.done_ticket, 1u);
+    // release: the block's atomics (ordered before this thread by the barrier above) are out before the ticket is
+    // taken; acquire: the block that draws the last ticket sees every other block's
+    unsigned t;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(t) : "l"(p.done_ticket) : "memory");
     sm.s_last = (t == (unsigned)(G - 1));
-    __threadfence();
   }
   __syncthreads();
   if (sm.s_last) {
